@@ -53,7 +53,8 @@ typedef enum {
 
 typedef enum { VXL_BF16 = 0, VXL_F32 = 1 } vxl_dtype;
 
-/* Relevance score of a chunk (the paper leaves the rule open: "attention score mechanism").
+/* Relevance score of a chunk (Bi-level KVs Decoding paragraph: the paper lists an attention-score
+ * rule among several possible ones and gives no formula).
  * VXL_SCORE_LSE   mean over query heads of ln sum_{p in sparse(c)} exp(scale * q.k_p)   (default)
  * VXL_SCORE_MASS  mean over query heads of the share of the head's softmax over the whole sparse
  *                 level that falls on the chunk: exp(lse[h,c]) / sum_c' exp(lse[h,c'])
@@ -97,8 +98,8 @@ typedef struct vxl_shape {
                                   vxl_bilevel_decode_attn when it selects itself              */
 } vxl_shape;
 
-/* The sparse level stored on its own (paper: "Both these dense and sparse KVs are then
- * stored"): k_sparse/v_sparse are [B, C*R, Hkv, D] bf16, contiguous, row c*R+r = the KV row
+/* The sparse level stored on its own (Bi-level KVs Decoding paragraph: both levels of every
+ * chunk are kept after prefill): k_sparse/v_sparse are [B, C*R, Hkv, D] bf16, contiguous, row c*R+r = the KV row
  * retained_idx[c][r].  Built by vxl_pack_retained.  Optional everywhere it appears. */
 typedef struct vxl_sparse_level {
     const void *k_sparse;
@@ -123,8 +124,8 @@ size_t vxl_workspace_bytes(int32_t op, const vxl_shape *shape, int32_t C, int32_
  * contiguous, may be NULL.  Requires T % chunk_len == 0; R may be 0 (retained_idx may then be
  * NULL).  bf16 products, fp32 accumulation and softmax.
  *
- * Sliding chunk window and prefix (same paragraph: "a sliding chunk window with a defined step
- * size", "the system prompt"; Fig. 2 right).  With S = shape->prefill_step (a divisor of
+ * Sliding chunk window and prefix (same paragraph and Fig. 2 right: the window advances by a
+ * step smaller than its length, and the system prompt stays visible).  With S = shape->prefill_step (a divisor of
  * chunk_len) and P0 = shape->prefix_len, the tokens after the prefix form blocks of S; a window
  * of chunk_len tokens advances by S, and the tokens it covers for the first time see the rest of
  * it.  For i >= P0, u = (i - P0) / S, ws = max(0, (u+1)*S - chunk_len):
@@ -139,7 +140,7 @@ vxl_status vxl_chunk_prefill_attn(const void *q, const void *k, const void *v,
 
 /*
  * Per-chunk relevance and top-k selection (paper: "Bi-level KVs Decoding" paragraph: a
- * relevance score per chunk, dense KVs for "several" highly relevant chunks).  The paper
+ * relevance score per chunk, dense KVs for the few most relevant chunks).  The paper
  * leaves the scoring rule open; this library implements the attention-score form on the
  * sparse level:
  *   scores[b,c] = (1/Hq) * sum_h  ln sum_{p in retained_idx[c]} exp( scale * q[b,h].k[b,p,g] )
@@ -158,8 +159,8 @@ vxl_status vxl_chunk_scores(const void *q, const void *k_cache,
                             void *cuda_stream);
 
 /*
- * Relevance for a query of several tokens (paper: the relevance oracle scores each chunk against
- * "a specific task query text"; how the tokens' scores are pooled is not stated).  This call takes
+ * Relevance for a query of several tokens (Bi-level KVs Decoding paragraph: chunks are scored
+ * against the text of the task query; how the tokens' scores are pooled is not stated).  This call takes
  * the arithmetic mean over the n_query_tokens tokens and the query heads of the same
  * log-sum-exp as vxl_chunk_scores:
  *   scores[b,c] = 1/(Tq*Hq) * sum_t sum_h ln sum_{p in sparse(c)} exp( scale * q[b,t,h].k[b,p,g] )
@@ -175,8 +176,8 @@ vxl_status vxl_chunk_scores_multi(const void *q, int32_t n_query_tokens, const v
                                   void *cuda_stream);
 
 /*
- * Selection from relevance scores computed elsewhere (paper: the relevance oracle "can be
- * implemented via various methods", e.g. an embedder or a custom pipeline): the `topk` chunks
+ * Selection from relevance scores computed elsewhere (Bi-level KVs Decoding paragraph: the scorer
+ * is left open, e.g. an embedding model or a pipeline of the user's own): the `topk` chunks
  * with the largest score per sequence, equal scores going to the lower chunk id, written as
  * ascending chunk ids.  scores [B,C] fp32 and topk_idx [B,topk] int32 are device memory; the
  * result can be passed as `selected` to vxl_bilevel_decode_attn.  C <= 4096.
@@ -223,14 +224,15 @@ vxl_status vxl_chunk_scores_static(const void *q, const void *k_cache,
 
 /*
  * Bi-level KV decoding attention (paper: "Bi-level KVs Decoding" paragraph, Fig. 3): one
- * query token per sequence attends over the "mixed KV" set = all rows
+ * query token per sequence attends over the mixed KV set = all rows
  * [off[c], off[c+1]) of the selected chunks plus the rows retained_idx[c] of every other
  * chunk (a chunk is read at one level only):
  *   out[b,h,:] = softmax over that set of scale * q[b,h].k  applied to v ;  lse[b,h] optional.
  * `selected` [B,topk] chunk ids (any order) chooses the dense chunks; NULL makes the call
  * score the chunks and pick the top-k itself (same rule as vxl_chunk_scores), in which case
  * scores_out [B,C] and topk_out [B,topk] receive them when non-NULL.  topk may be 0..C.
- * max_chunk_len >= max_c (off[c+1]-off[c]) sizes the launch (longer chunks stay correct).
+ * max_chunk_len must bound every selected chunk: it sizes the launch and the workspace; a selected
+ * chunk that is longer is cut off there and sets the status word to VXL_ERR_INVALID_ARG.
  * out [B,Hq,D] (out strides of `shape`, out_stride_t unused).
  */
 vxl_status vxl_bilevel_decode_attn(const void *q, const void *k_cache, const void *v_cache,
@@ -243,9 +245,9 @@ vxl_status vxl_bilevel_decode_attn(const void *q, const void *k_cache, const voi
                                    void *cuda_stream);
 
 /*
- * Bi-level KV decoding with the dense level kept off the device (paper: "Both these dense and
- * sparse KVs are then stored in an offline memory"; the strategy "selectively loads KVs for each
- * video chunk": dense KVs for the relevant ones, sparse KVs for the rest).  Here the sparse level
+ * Bi-level KV decoding with the dense level kept off the device (Bi-level KVs Decoding paragraph:
+ * both levels are parked in memory outside the accelerator and reloaded per query, dense KVs for
+ * the relevant chunks, sparse KVs for the rest).  Here the sparse level
  * lives on the device and the dense cache in pinned host memory; one call
  *   1. scores the chunks on the sparse level and picks the top-k (as vxl_chunk_scores),
  *   2. brings the selection to the host -- THIS CALL SYNCHRONISES cuda_stream at that point --
@@ -283,11 +285,11 @@ vxl_status vxl_pack_retained(const void *k_cache, const void *v_cache,
                              const vxl_shape *shape, void *cuda_stream);
 
 /*
- * Sparse level by pooling (paper: "For each resulting KV chunk, we then apply a pooling
- * operation to generate corresponding sparse KVs").  The paper does not name the pooling; this
+ * Sparse level by pooling (Bi-level KVs Decoding paragraph: each chunk's sparse KVs come from a
+ * pooling step over its dense ones).  The paper does not name the pooling; this
  * call averages: pooled row r of chunk c is the mean of the dense rows
  * [off[c] + r*len/R, off[c] + (r+1)*len/R) (integer division, len = off[c+1] - off[c]; an empty
- * window gives a zero row), summed and divided in fp32 and stored as bf16.
+ * window gives a zero row), summed and divided in fp64 and rounded once to bf16.
  * k_cache/v_cache [B,T,Hkv,D]; chunk_offsets [C+1] (device); k_sparse/v_sparse [B, C*R, Hkv, D]
  * bf16, contiguous: a vxl_sparse_level for vxl_chunk_scores / vxl_bilevel_decode_attn, which
  * then read R pooled rows for a chunk that is not selected (retained_idx may be NULL there).

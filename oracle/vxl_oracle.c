@@ -9,11 +9,11 @@
  * What it follows (Efficiency Optimization subsection of the paper):
  *   - Chunk-based pre-filling paragraph and Fig. 2 (left): a token of chunk c attends to the
  *     tokens of its own chunk (causally, since the language model is decoder-only) and to the
- *     retained KVs ("historical timestamp tokens") of every preceding chunk.
+ *     retained KVs (the KVs of the timestamp tokens met so far) of every preceding chunk.
  *   - Bi-level KVs decoding paragraph and Fig. 3: every chunk has a dense level (all its KVs)
  *     and a sparse level (a sub-sampled set of them); a relevance score is computed per chunk;
  *     the most relevant chunks are read dense, the others sparse; the rows read are
- *     concatenated into one "mixed KV" set over which the query attends.
+ *     concatenated into one mixed KV set over which the query attends.
  * Given the key set, the result is ordinary softmax attention, so each function below is that
  * definition written out: explicit mask row / explicit score table / explicit mixed row list,
  * softmax by max-subtraction, all sums in double.  Inputs are bf16 bit patterns widened
@@ -140,10 +140,10 @@ int vxl_oracle_prefill(const uint16_t *q, const uint16_t *k, const uint16_t *v,
 }
 
 /*
- * Chunk-based pre-filling with a sliding chunk window and an always-visible prefix (paragraph
- * "Chunk-based Pre-filling": the current chunk attends "to itself, historical timestamp tokens
- * and the system prompt"; "a sliding chunk window with a defined step size" lets it "attend to
- * overlapping portion of the preceding chunk's detailed visual information"; Fig. 2 right).
+ * Chunk-based pre-filling with a sliding chunk window and an always-visible prefix (Chunk-based
+ * Pre-filling paragraph and Fig. 2 right: besides itself and the earlier timestamp tokens, the
+ * current chunk sees the system prompt, and because the window moves by a step shorter than the
+ * window it also sees the dense tokens of the part of the previous chunk that it overlaps).
  *
  * Reading (the paper gives no formula): the first P0 tokens are the prefix.  The other tokens are
  * cut into step blocks of S tokens.  A window of L tokens (L a multiple of S) slides by S; the
@@ -206,8 +206,8 @@ int vxl_oracle_prefill_window(const uint16_t *q, const uint16_t *k, const uint16
 }
 
 /*
- * Per-chunk relevance (paragraph "Bi-level KVs Decoding": "computes a relevance score for
- * each video input chunk"; the attention-score form is one of the options the paper lists and
+ * Per-chunk relevance (Bi-level KVs Decoding paragraph: every video chunk gets a
+ * relevance score for the query; the attention-score form is one of the options the paper lists and
  * the formula is this build's reading):
  *   lse_hc[h, c] = ln sum_{p in retained_idx[c]} exp(scale * q[h].k[p, g(h)])
  *   scores[c]    = (1/Hq) * sum_h lse_hc[h, c]
@@ -250,7 +250,7 @@ int vxl_oracle_scores(const uint16_t *q, const uint16_t *k, int T, int Hq, int H
 }
 
 /*
- * Top-k chunk selection ("loads dense KVs for several video chunks that are highly relevant").
+ * Top-k chunk selection (Bi-level KVs Decoding paragraph: the few most relevant chunks are read dense).
  * The k largest scores; equal scores go to the lower chunk index (a reading: the paper gives
  * no tie rule).  Selection by repeated arg-max so the rule is visible; output ascending chunk
  * ids.  *gap = (k-th largest) - ((k+1)-th largest), +inf if k == 0 or k == C.
@@ -279,8 +279,8 @@ int vxl_oracle_topk(const double *scores, int C, int k, int32_t *idx_out, double
 }
 
 /*
- * Mixed-KV decode attention (paragraph "Bi-level KVs Decoding": dense KVs for the selected
- * chunks, sparse KVs for the others, "concatenated to form a new, complete mixed KV set").
+ * Mixed-KV decode attention (Bi-level KVs Decoding paragraph: dense KVs for the selected
+ * chunks, sparse KVs for the others, joined into one mixed KV set that replaces the full cache).
  * The explicit row list is built chunk by chunk: all rows [off[c], off[c+1]) when c is in
  * `selected`, else the rows retained_idx[c].  A chunk is read at one level only.
  * One sequence: q [Hq,D], k/v [T,Hkv,D].  mixed_rows_out (nullable) receives the list,
@@ -332,8 +332,8 @@ int vxl_oracle_decode(const uint16_t *q, const uint16_t *k, const uint16_t *v,
 }
 
 /*
- * Sparse level by pooling (paragraph "Bi-level KVs Decoding": "For each resulting KV chunk, we
- * then apply a pooling operation to generate corresponding sparse KVs").  Reading: average
+ * Sparse level by pooling (Bi-level KVs Decoding paragraph: the sparse KVs of a chunk are made by
+ * pooling its dense KVs; the kind of pooling is not named).  Reading: average
  * pooling, R pooled rows per chunk; pooled row r of chunk c is the arithmetic mean of the dense
  * rows [lo + floor(r*len/R), lo + floor((r+1)*len/R)) with lo = chunk_offsets[c] and
  * len = chunk_offsets[c+1] - lo (equal windows of len/R rows when R divides len; an empty window
@@ -431,8 +431,8 @@ int vxl_oracle_decode_levels(const uint16_t *q, const uint16_t *k, const uint16_
 }
 
 /*
- * Relevance for a query of several tokens (the paper scores chunks against "a specific task query
- * text", i.e. more than one token; how token scores are pooled is not stated).  Reading: the
+ * Relevance for a query of several tokens (the paper scores chunks against the text of the task
+ * query, i.e. more than one token; how token scores are pooled is not stated).  Reading: the
  * score of a chunk is the arithmetic mean, over the query tokens and the query heads, of the
  * same log-sum-exp as above.
  *   q [Tq,Hq,D]; scores [C].  Tq == 1 is vxl_oracle_scores.
@@ -456,7 +456,7 @@ int vxl_oracle_scores_multi(const uint16_t *q, int Tq, const uint16_t *k, int T,
 }
 
 /*
- * Relevance as attention mass (another "attention score mechanism" reading of the paper's
+ * Relevance as attention mass (another attention-score reading of the paper's
  * relevance oracle): the share of the query's softmax attention over the whole sparse level that
  * falls on the chunk's sparse rows, averaged over the query heads:
  *   mass[h, c] = sum_{p in sparse(c)} exp(x_hp) / sum_{all sparse p'} exp(x_hp')

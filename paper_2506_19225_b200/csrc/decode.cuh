@@ -647,9 +647,11 @@ __global__ void __launch_bounds__(1024) topk_scores_kernel(const float *__restri
 
 // ---------------------------------------------------------------------------------------
 // Sparse level by average pooling: pooled row r of chunk c = mean of the dense rows
-// [lo + r*len/R, lo + (r+1)*len/R) (integer division), summed in fp32 in row order, divided in
-// fp32 and rounded once to bf16.  One thread per (sequence, pooled row, 16-byte column piece);
-// the threads of a warp read 512 contiguous bytes of every row of the window.
+// [lo + r*len/R, lo + (r+1)*len/R) (integer division), summed in fp64 in row order, divided in
+// fp64 and rounded once to bf16 (the pass is bound by HBM; the wide arithmetic is free and makes
+// the stored bytes a function of the inputs alone, with no second rounding).  One thread per
+// (sequence, pooled row, 16-byte column piece); the threads of a warp read 512 contiguous bytes
+// of every row of the window.
 struct PoolParams {
     const __nv_bfloat16 *k, *v;
     __nv_bfloat16 *ks, *vs;
@@ -658,6 +660,16 @@ struct PoolParams {
     int64_t kv_sb, kv_st, kv_sh;
     int B, T, Hkv, D, C, R;
 };
+
+// fp64 -> bf16 with a single round-to-nearest-even: the value is first cut to fp32 by truncation
+// with a sticky last bit (round to odd), which keeps enough information for the final rounding
+// of the 24-bit significand to 8 bits to be the rounding of the fp64 value itself.
+__device__ __forceinline__ float f64_to_f32_round_to_odd(double x)
+{
+    float f = __double2float_rz(x);
+    if ((double)f != x) f = __uint_as_float(__float_as_uint(f) | 1u);
+    return f;
+}
 
 __global__ void __launch_bounds__(256) pool_sparse_kernel(const PoolParams p)
 {
@@ -675,9 +687,9 @@ __global__ void __launch_bounds__(256) pool_sparse_kernel(const PoolParams p)
         const int a = lo + (int)(((int64_t)r * len) / p.R), z = lo + (int)(((int64_t)(r + 1) * len) / p.R);
         const int hh = piece / (p.D / 8), dd = (piece % (p.D / 8)) * 8;
         const int64_t col = (int64_t)b * p.kv_sb + (int64_t)hh * p.kv_sh + dd;
-        float sk[8], sv[8];
+        double sk[8], sv[8];
 #pragma unroll
-        for (int x = 0; x < 8; ++x) sk[x] = sv[x] = 0.f;
+        for (int x = 0; x < 8; ++x) sk[x] = sv[x] = 0.0;
         for (int j = a; j < z; ++j) {
             // read once: streaming loads (evict-first) leave the rest of L2 alone
             const uint4 uk = __ldcs(reinterpret_cast<const uint4 *>(p.k + col + (int64_t)j * p.kv_st));
@@ -687,17 +699,17 @@ __global__ void __launch_bounds__(256) pool_sparse_kernel(const PoolParams p)
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const float2 fk = __bfloat1622float2(bk[x]), fv = __bfloat1622float2(bv[x]);
-                sk[2 * x] += fk.x; sk[2 * x + 1] += fk.y;
-                sv[2 * x] += fv.x; sv[2 * x + 1] += fv.y;
+                sk[2 * x] += (double)fk.x; sk[2 * x + 1] += (double)fk.y;
+                sv[2 * x] += (double)fv.x; sv[2 * x + 1] += (double)fv.y;
             }
         }
-        const float n = (float)(z - a);
+        const double n = (double)(z - a);
         uint4 ok, ov;
         uint32_t *wk = reinterpret_cast<uint32_t *>(&ok), *wv = reinterpret_cast<uint32_t *>(&ov);
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-            wk[x] = (z > a) ? pack_bf16(sk[2 * x] / n, sk[2 * x + 1] / n) : 0u;
-            wv[x] = (z > a) ? pack_bf16(sv[2 * x] / n, sv[2 * x + 1] / n) : 0u;
+            wk[x] = (z > a) ? pack_bf16(f64_to_f32_round_to_odd(sk[2 * x] / n), f64_to_f32_round_to_odd(sk[2 * x + 1] / n)) : 0u;
+            wv[x] = (z > a) ? pack_bf16(f64_to_f32_round_to_odd(sv[2 * x] / n), f64_to_f32_round_to_odd(sv[2 * x + 1] / n)) : 0u;
         }
         const int64_t dst = (e * p.Hkv + hh) * p.D + dd;
         *reinterpret_cast<uint4 *>(p.ks + dst) = ok;

@@ -335,6 +335,16 @@ decode_stream_kernel(const __grid_constant__ StreamMaps maps, const StreamParams
                                                   ((((col & 63) >> 3) ^ (key & 7)) << 4);
                             uint32_t b0, b1, b2, b3;
                             ldsm_x4_t(addr, b0, b1, b2, b3);
+                            if (nvalid < TK) {
+                                // Rows past the item's end are whatever follows in memory (the next chunk, unwritten
+                                // cache capacity, a staging slot's leftovers): their probabilities are 0, and 0 x NaN
+                                // must not reach O, so those V rows are read as zeros.  b0/b2 hold keys kg*16 + 2t, +1
+                                // and b1/b3 keys kg*16 + 8 + 2t, +1 (low half first).
+                                const int k0 = kg * 16 + 2 * t;
+                                const uint32_t m0 = (k0 < nvalid ? 0xFFFFu : 0u) | (k0 + 1 < nvalid ? 0xFFFF0000u : 0u);
+                                const uint32_t m1 = (k0 + 8 < nvalid ? 0xFFFFu : 0u) | (k0 + 9 < nvalid ? 0xFFFF0000u : 0u);
+                                b0 &= m0; b2 &= m0; b1 &= m1; b3 &= m1;
+                            }
                             mma_bf16(o[2 * nd2], a0, a1, a2, a3, b0, b1);
                             mma_bf16(o[2 * nd2 + 1], a0, a1, a2, a3, b2, b3);
                         }
@@ -521,7 +531,7 @@ __global__ void __launch_bounds__(1024) combine_fast_kernel(const CombineParams 
 // memory): pass A, one thread per slot, finds the largest partial maximum among the live slots and
 // turns every slot into a weight 2^(m - max) (0 for empty slots and for sparse slots of chunks
 // that were read dense); pass B sums weight * partial output with all loads of a thread in flight.
-constexpr int kCombineMaxSlots = 8192;
+constexpr int kCombineMaxSlots = 8000;     // weights (4 B each) + 16.5 KB of static shared memory stay under 48 KB
 
 template <int D>
 __global__ void __launch_bounds__(1024) combine_two_pass_kernel(const CombineParams p)

@@ -303,6 +303,19 @@ vxl_status check_decode_common(const vxl_shape *s, const void *q, const void *k,
     return VXL_OK;
 }
 
+// Host-side argument checks of vxl_chunk_scores (everything but the workspace).
+vxl_status check_scores_args(const vxl_shape *s, const void *q, const void *k, const int32_t *off, int C,
+                             const int32_t *ridx, int R, int64_t ridx_sb, const vxl_sparse_level *sp,
+                             const float *scores, int topk)
+{
+    const vxl_status vs = check_decode_common(s, q, k, off, C, ridx, R, ridx_sb, sp, false);
+    if (vs != VXL_OK) return vs;
+    if (scores == nullptr || topk < 0 || topk > C) return VXL_ERR_INVALID_ARG;
+    if (C > kMaxChunks) return VXL_ERR_UNSUPPORTED;
+    if (R > 0 && ridx == nullptr && (sp == nullptr || (int64_t)s->B * C * R >= (1ll << 31))) return VXL_ERR_INVALID_ARG;
+    return VXL_OK;
+}
+
 cudaError_t launch_validate(const int32_t *ridx, const int32_t *off, WsHeader *hdr, int64_t ridx_sb, int nb,
                             int C, int R, int L, int T, cudaStream_t st, int base = 0)
 {
@@ -565,10 +578,8 @@ vxl_status vxl_chunk_scores(const void *q, const void *k_cache, const int32_t *c
                             const vxl_sparse_level *sparse, float *scores, int32_t topk, int32_t *topk_idx,
                             const vxl_shape *s, void *workspace, size_t ws_bytes, void *cuda_stream)
 {
-    vxl_status vs = check_decode_common(s, q, k_cache, chunk_offsets, C, retained_idx, R, ridx_stride_b, sparse, false);
+    vxl_status vs = check_scores_args(s, q, k_cache, chunk_offsets, C, retained_idx, R, ridx_stride_b, sparse, scores, topk);
     if (vs != VXL_OK) return vs;
-    if (scores == nullptr || topk < 0 || topk > C) return VXL_ERR_INVALID_ARG;
-    if (C > kMaxChunks) return VXL_ERR_UNSUPPORTED;
     if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         ws_bytes < vxl_workspace_bytes(VXL_OP_SCORES, s, C, R, 0, 0))
         return VXL_ERR_WORKSPACE;
@@ -642,11 +653,14 @@ vxl_status vxl_chunk_scores_static(const void *q, const void *k_cache, const int
                                    const vxl_sparse_level *sparse, float *scores, int32_t topk, int32_t *topk_idx,
                                    int32_t *device_status_out, const vxl_shape *s, void *cuda_stream)
 {
-    // Size check first: a problem that does not fit is refused before anything is touched.
+    // Every host-side check comes first: a call that is refused has touched neither the stream nor the
+    // shared array (whose status word an earlier call's status copy may not have read yet).
     if (!shape_ok(s) || C <= 0 || R < 0) return VXL_ERR_INVALID_ARG;
     const size_t need = vxl_workspace_bytes(VXL_OP_SCORES, s, C, R, 0, 0);
     if (need == 0) return VXL_ERR_INVALID_ARG;
     if (need > kStaticScratchBytes) return VXL_ERR_WORKSPACE;
+    const vxl_status pre = check_scores_args(s, q, k_cache, chunk_offsets, C, retained_idx, R, ridx_stride_b, sparse, scores, topk);
+    if (pre != VXL_OK) return pre;
     void *scratch = static_scratch_address();
     if (scratch == nullptr) return VXL_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

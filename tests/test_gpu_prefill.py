@@ -144,7 +144,7 @@ def test_kernel_kind_selection():
     assert vb.prefill_kernel_kind(B=1, T=100, Hq=2, Hkv=1, D=64, chunk_len=64, R=0) == -1
 
 
-@pytest.mark.parametrize("name", ["cfg2_16k", "cfg3_64k", "sweep_L512", "sweep_L4096"])
+@pytest.mark.parametrize("name", ["cfg2_16k", "cfg3_64k", "sweep_L512", "sweep_L1024", "sweep_L2048", "sweep_L4096"])
 def test_full_size_sampled(name):
     case = inputs.make_prefill(name)
     rows = sample_rows(case.T, case.L, 24, seed=case.seed)
@@ -162,8 +162,16 @@ def test_cfg2_general_kernel_sampled():
 
 
 def test_cfg4_256k_sampled():
+    """262,144 tokens: chunks 0, 1, 2, 63, 126 and 127 compared in full (every row, every head), 64 seeded
+    rows of every other chunk, plus the tile and chunk boundaries of `sample_rows`: 7.7 % of all rows."""
     case = inputs.make_prefill("cfg4_256k")
-    rows = sample_rows(case.T, case.L, 16, seed=case.seed)
+    rng = np.random.default_rng(case.seed + 1)
+    full = (0, 1, 2, 63, 126, 127)
+    parts = [np.arange(c * case.L, (c + 1) * case.L) for c in full]
+    parts += [c * case.L + np.sort(rng.choice(case.L, size=64, replace=False)) for c in range(case.C) if c not in full]
+    parts.append(sample_rows(case.T, case.L, 16, seed=case.seed))
+    rows = np.unique(np.concatenate(parts)).astype(np.int32)
+    assert rows.size >= 6 * case.L + 64 * (case.C - 6)
     compare_sampled(case, rows)
 
 

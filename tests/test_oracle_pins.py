@@ -434,6 +434,18 @@ def test_pool_hand_values_and_rounding_to_nearest_even():
     np.testing.assert_array_equal(got[:, 0, 0], [1.5, 4.0])
 
 
+def test_pool_rounding_in_the_subnormal_range_of_bf16():
+    # bf16 below 2^-126 counts in units of 2^-133 (bit patterns 0x0001 .. 0x007f).  Means of two rows, by hand:
+    #   (3u, 2u) -> 2.5u: tie, even wins -> 2u        (3u, 4u) -> 3.5u: tie -> 4u
+    #   (127u, 128u) -> 127.5u: tie -> 128u = the smallest normal 0x0080 (the encoding runs on)
+    #   (-1u, -2u) -> -1.5u: tie -> -2u               (1u, 0) -> 0.5u: tie -> 0
+    #   (5u, 2u) -> 3.5u -> 4u ; (6u, 1u) -> 3.5u -> 4u ; (1u, 2u) -> 1.5u -> 2u
+    rows = np.array([[0x0003, 0x0003, 0x007F, 0x8001, 0x0001, 0x0005, 0x0006, 0x0001],
+                     [0x0002, 0x0004, 0x0080, 0x8002, 0x0000, 0x0002, 0x0001, 0x0002]], dtype=np.uint16)
+    got = ref.pool(rows.reshape(2, 1, 8), np.array([0, 2], dtype=np.int32), 1).reshape(-1)
+    assert got.tolist() == [0x0002, 0x0004, 0x0080, 0x8002, 0x0000, 0x0004, 0x0004, 0x0002]
+
+
 def test_pool_matches_numpy_mean_within_half_an_ulp():
     d = small_decode(T=256, L=64, R=4)
     got = inputs.bf16_bits_to_f64(ref.pool(d.v[1], d.chunk_offsets, 8))

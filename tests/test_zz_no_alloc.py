@@ -17,7 +17,8 @@ import torch
 
 from paper_2506_19225_b200 import binding as vb
 from paper_2506_19225_b200 import inputs
-from tests.parity import LSE_ABS_ERR, to_gpu
+from oracle import ref
+from tests.parity import LSE_ABS_ERR, TOPK_NEAR_TIE, to_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -44,9 +45,16 @@ def _compare(prob):
                            scale=d.scale, sparse=sparse)
     torch.cuda.synchronize()
     assert int(status.item()) == vb.VXL_OK
-    err = (scores - want_scores).abs().max().item()
-    assert err <= LSE_ABS_ERR, f"scores differ by {err:.3e}"
+    # the two entry points run the same kernels on the same inputs: equal bit for bit, not merely close
+    assert torch.equal(scores, want_scores)
     assert torch.equal(topk_idx, want_topk)
+    # and the answer is the right one: the fp64 oracle on the same bytes
+    for b in range(d.B):
+        _, sc = ref.scores(d.q[b], d.k[b], d.retained_idx, d.scale)
+        idx, gap = ref.topk(sc, topk)
+        err = np.abs(scores[b].double().cpu().numpy() - sc).max()
+        assert err <= LSE_ABS_ERR, f"scores differ from the oracle by {err:.3e}"
+        assert topk_idx[b].cpu().tolist() == idx.tolist() or gap < TOPK_NEAR_TIE
 
 
 def test_static_scratch_matches_workspace_call_twice_in_a_row():
@@ -71,3 +79,30 @@ def test_static_scratch_refuses_problems_beyond_its_size():
                                      vb._ptr(scores), 0, None, None, ctypes.byref(shape), vb._stream())
     assert rc == vb.VXL_ERR_WORKSPACE
     torch.cuda.synchronize()
+
+
+def test_static_scratch_reports_a_bad_index_and_a_refused_call_touches_nothing():
+    d, q, k, off, ridx, sparse, topk = _problem(B=2, T=2048, L=128, R=16, topk=3, seed=43, packed=False)
+    scores = torch.zeros((d.B, d.C), dtype=torch.float32, device="cuda")
+    topk_idx = torch.zeros((d.B, topk), dtype=torch.int32, device="cuda")
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    bad = ridx.clone()
+    bad[1, 2] = d.T + 5                      # outside its chunk and the cache: clamped when read, reported under validate
+    vb.chunk_scores_static(q, k, off, bad, scores, topk=topk, topk_idx=topk_idx, device_status=status,
+                           scale=d.scale, validate=True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == vb.VXL_ERR_INVALID_INDEX
+    # a call refused on the host (topk > C) enqueues nothing: the status word of the call before it is still there
+    lib = vb.load()
+    shape = vb._decode_shape(q, k, None, None, False)
+    rc = lib.vxl_chunk_scores_static(vb._ptr(q), vb._ptr(k), vb._ptr(off), d.C, vb._ptr(ridx), d.R, 0, None,
+                                     vb._ptr(scores), d.C + 1, vb._ptr(topk_idx), vb._ptr(status),
+                                     ctypes.byref(shape), vb._stream())
+    assert rc == vb.VXL_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert int(status.item()) == vb.VXL_ERR_INVALID_INDEX
+    # the next good call starts from a clean status word
+    vb.chunk_scores_static(q, k, off, ridx, scores, topk=topk, topk_idx=topk_idx, device_status=status, scale=d.scale,
+                           validate=True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == vb.VXL_OK
