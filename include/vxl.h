@@ -19,6 +19,7 @@
  *   Stream     `cuda_stream` is a cudaStream_t (NULL = legacy default stream).  Calls only
  *              enqueue work; they never synchronise, except vxl_device_status and
  *              vxl_bilevel_decode_offline (which needs the selection on the host).
+ *              vxl_chunk_prefill_host takes HOST arrays beside the device ones (stated there).
  *   Workspace  caller-allocated scratch of at least vxl_workspace_bytes(...) bytes, 256-byte
  *              aligned, zero-filled once before its first use (cudaMemset).  Its first word is
  *              a sticky device status (0 = ok).  Calls that run concurrently on different
@@ -137,6 +138,36 @@ vxl_status vxl_chunk_prefill_attn(const void *q, const void *k, const void *v,
                                   int32_t chunk_len, const int32_t *retained_idx, int32_t R,
                                   void *out, float *lse, const vxl_shape *shape,
                                   void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Chunk-based pre-filling of sequences whose tokens live in HOST memory (Chunk-based Pre-filling
+ * paragraph: the long input is encoded one chunk after the other, each step touching only the
+ * current chunk and the few retained KVs before it).  The call runs the chunks as a pipeline over
+ * three streams: the rows of chunk group g travel host -> device on h2d_stream, group g is attended
+ * on cuda_stream by vxl_chunk_prefill_attn restricted to its blocks (nothing after the group is
+ * read), and its output rows travel device -> host on d2h_stream, so copies in both directions
+ * overlap the kernels and each other.  One 2-D copy per tensor and group (its rows in every
+ * sequence).  Same result as vxl_chunk_prefill_attn over the same data.
+ *   q_host [B,T,Hq,D], k_host/v_host [B,T,Hkv,D] bf16, retained_idx_host [C,R] int32, out_host
+ *   [B,T,Hq,D] of shape->out_dtype, lse_host [B,T,Hq] fp32 or NULL: HOST memory, contiguous; pin it
+ *   (cudaHostAlloc / cudaHostRegister), or the copies will not overlap anything.
+ *   q_dev, k_dev, v_dev, retained_idx_dev, out_dev, lse_dev (NULL iff lse_host is): DEVICE arrays of
+ *   the same shapes, caller-owned, overwritten; they hold the sequence afterwards (k_dev/v_dev are
+ *   the KV cache the decoding calls read).
+ *   chunks_per_call: chunks per pipeline step (0 = 1).  The strides in `shape` must describe the
+ *   contiguous layout; plain chunks only (no window, prefix or block range).
+ * The three streams must differ.  On return everything is enqueued; work submitted to cuda_stream
+ * afterwards is ordered after the last copy back, and the host arrays may be read once
+ * cuda_stream (or d2h_stream) has been synchronised.  The library keeps a pool of CUDA events per
+ * device for this call (created on first use, never during stream capture).
+ */
+vxl_status vxl_chunk_prefill_host(const void *q_host, const void *k_host, const void *v_host,
+                                  int32_t chunk_len, const int32_t *retained_idx_host, int32_t R,
+                                  void *out_host, float *lse_host,
+                                  void *q_dev, void *k_dev, void *v_dev, int32_t *retained_idx_dev,
+                                  void *out_dev, float *lse_dev, int32_t chunks_per_call,
+                                  const vxl_shape *shape, void *workspace, size_t ws_bytes,
+                                  void *cuda_stream, void *h2d_stream, void *d2h_stream);
 
 /*
  * Per-chunk relevance and top-k selection (paper: "Bi-level KVs Decoding" paragraph: a

@@ -22,7 +22,7 @@ VXL_BF16, VXL_F32 = 0, 1
 VXL_OP_PREFILL, VXL_OP_SCORES, VXL_OP_DECODE = 0, 1, 2
 VXL_SCORE_LSE, VXL_SCORE_MASS = 0, 1
 
-EXPORTS = ("vxl_workspace_bytes", "vxl_chunk_prefill_attn", "vxl_chunk_scores",
+EXPORTS = ("vxl_workspace_bytes", "vxl_chunk_prefill_attn", "vxl_chunk_prefill_host", "vxl_chunk_scores",
            "vxl_chunk_scores_static", "vxl_chunk_scores_multi", "vxl_topk_select", "vxl_bilevel_decode_attn", "vxl_bilevel_decode_offline", "vxl_pack_retained", "vxl_pool_sparse", "vxl_device_status",
            "vxl_status_str", "vxl_prefill_kernel_kind")
 
@@ -72,6 +72,9 @@ def load():
         lib.vxl_chunk_prefill_attn.restype = ctypes.c_int
         lib.vxl_chunk_prefill_attn.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp, ctypes.POINTER(VxlShape),
                                                vp, sz, vp]
+        lib.vxl_chunk_prefill_host.restype = ctypes.c_int
+        lib.vxl_chunk_prefill_host.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32,
+                                               ctypes.POINTER(VxlShape), vp, sz, vp, vp, vp]
         lib.vxl_chunk_scores.restype = ctypes.c_int
         lib.vxl_chunk_scores.argtypes = [vp, vp, vp, i32, vp, i32, i64, ctypes.POINTER(VxlSparseLevel),
                                          vp, i32, vp, ctypes.POINTER(VxlShape), vp, sz, vp]
@@ -397,69 +400,54 @@ def bilevel_decode_attn(q, k_cache, v_cache, chunk_offsets, retained_idx, topk: 
 
 
 class HostPrefill:
-    """Chunk-based pre-filling of one sequence whose tokens live in pinned host memory.
+    """Chunk-based pre-filling of sequences whose tokens live in pinned host memory
+    (vxl_chunk_prefill_host: copy chunk c in, attend chunk c, copy its output rows back, on three
+    streams).  This class only holds what the call needs (device arrays, workspace, two copy streams),
+    so that ``run`` allocates nothing; the pipeline itself is inside the library."""
 
-    The chunks go through three streams: copy chunk c in, attend chunk c (vxl_chunk_prefill_attn
-    over the block range of that chunk), copy its output rows back, so that the copies in both
-    directions overlap the kernels and each other.  All device buffers, streams and events are
-    made here; ``run`` allocates nothing."""
-
-    def __init__(self, T: int, Hq: int, Hkv: int, D: int, chunk_len: int, R: int, *, device="cuda",
-                 out_dtype=torch.float32, chunks_per_call: int = 1, scale=None, force_general=False):
+    def __init__(self, T: int, Hq: int, Hkv: int, D: int, chunk_len: int, R: int, *, B: int = 1, device="cuda",
+                 out_dtype=torch.float32, chunks_per_call: int = 1, scale=None, force_general=False, with_lse=False):
         if T % chunk_len:
             raise ValueError("T must be a multiple of chunk_len")
-        self.T, self.Hq, self.Hkv, self.D, self.L, self.R = T, Hq, Hkv, D, chunk_len, R
+        self.B, self.T, self.Hq, self.Hkv, self.D, self.L, self.R = B, T, Hq, Hkv, D, chunk_len, R
         self.C = T // chunk_len
         self.per_call = max(1, int(chunks_per_call))
-        self.scale, self.force_general = scale, force_general
-        self.q = torch.empty((1, T, Hq, D), dtype=torch.bfloat16, device=device)
-        self.k = torch.empty((1, T, Hkv, D), dtype=torch.bfloat16, device=device)
+        self.q = torch.empty((B, T, Hq, D), dtype=torch.bfloat16, device=device)
+        self.k = torch.empty((B, T, Hkv, D), dtype=torch.bfloat16, device=device)
         self.v = torch.empty_like(self.k)
-        self.out = torch.empty((1, T, Hq, D), dtype=out_dtype, device=device)
-        self.ridx = torch.empty((self.C, R), dtype=torch.int32, device=device) if R > 0 else None
-        self.ws = prefill_workspace(B=1, T=T, Hq=Hq, Hkv=Hkv, D=D, chunk_len=chunk_len, R=R, device=device)
+        self.out = torch.empty((B, T, Hq, D), dtype=out_dtype, device=device)
+        self.lse = torch.empty((B, T, Hq), dtype=torch.float32, device=device) if with_lse else None
+        self.ridx = torch.empty((self.C, max(R, 1)), dtype=torch.int32, device=device)
+        self.ws = prefill_workspace(B=B, T=T, Hq=Hq, Hkv=Hkv, D=D, chunk_len=chunk_len, R=R, device=device)
         self.s_in, self.s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
-        n = (self.C + self.per_call - 1) // self.per_call
-        self.ev_in = [torch.cuda.Event() for _ in range(n)]
-        self.ev_done = [torch.cuda.Event() for _ in range(n)]
+        self.shape = make_shape(B=B, T=T, Hq=Hq, Hkv=Hkv, D=D, q_strides=(T * Hq * D, Hq * D, D),
+                                kv_strides=(T * Hkv * D, Hkv * D, D), scale=scale or 0.0,
+                                out_dtype=_out_code(out_dtype), force_general=force_general)
 
-    def run(self, q_host, k_host, v_host, retained_idx_host, out_host):
-        """q_host [T,Hq,D], k_host/v_host [T,Hkv,D]: pinned bf16 (or int16 bit patterns); retained_idx_host
-        [C,R] int32 pinned; out_host [T,Hq,D] pinned, of the output dtype.  Returns out_host; the copies
-        into it are ordered before later work on the current stream (synchronise it before reading)."""
-        for name, h, shp in (("q_host", q_host, (self.T, self.Hq, self.D)), ("k_host", k_host, (self.T, self.Hkv, self.D)),
-                             ("v_host", v_host, (self.T, self.Hkv, self.D)), ("out_host", out_host, (self.T, self.Hq, self.D))):
-            if tuple(h.shape) != shp or not h.is_pinned() or not h.is_contiguous():
-                raise ValueError(f"{name} must be a contiguous pinned host tensor of shape {shp}")
+    def run(self, q_host, k_host, v_host, retained_idx_host, out_host, lse_host=None, stream=None):
+        """q_host [B,T,Hq,D] (or [T,Hq,D] when B = 1), k_host/v_host likewise with Hkv: pinned bf16 (or their
+        bits as int16); retained_idx_host [C,R] int32; out_host pinned, of the output dtype.  Returns
+        out_host; the copies into it are ordered before later work on the stream (synchronise it before
+        reading)."""
+        B, T = self.B, self.T
+        for name, h, heads in (("q_host", q_host, self.Hq), ("k_host", k_host, self.Hkv), ("v_host", v_host, self.Hkv),
+                               ("out_host", out_host, self.Hq)):
+            if h.numel() != B * T * heads * self.D or not h.is_pinned() or not h.is_contiguous():
+                raise ValueError(f"{name} must be a contiguous pinned host tensor of {B} x {T} x {heads} x {self.D} elements")
         if q_host.element_size() != 2 or k_host.element_size() != 2 or v_host.element_size() != 2:
             raise ValueError("q_host / k_host / v_host hold bf16 values (torch.bfloat16, or their bits as int16)")
         if out_host.dtype != self.out.dtype:
             raise ValueError("out_host must have the output dtype")
-        main = torch.cuda.current_stream()
-        qd, kd, vd = (x[0].view(h.dtype) for x, h in ((self.q, q_host), (self.k, k_host), (self.v, v_host)))
-        self.s_in.wait_stream(main)                       # earlier kernels may still read the device buffers
-        self.s_out.wait_stream(main)
-        groups = [(c0, min(self.per_call, self.C - c0)) for c0 in range(0, self.C, self.per_call)]
-        with torch.cuda.stream(self.s_in):
-            if self.ridx is not None:
-                self.ridx.copy_(retained_idx_host, non_blocking=True)
-            for g, (c0, n) in enumerate(groups):
-                rows = slice(c0 * self.L, (c0 + n) * self.L)
-                qd[rows].copy_(q_host[rows], non_blocking=True)
-                kd[rows].copy_(k_host[rows], non_blocking=True)
-                vd[rows].copy_(v_host[rows], non_blocking=True)
-                self.ev_in[g].record(self.s_in)
-        for g, (c0, n) in enumerate(groups):
-            main.wait_event(self.ev_in[g])
-            chunk_prefill_attn(self.q, self.k, self.v, self.L, self.ridx, scale=self.scale, out=self.out,
-                               workspace=self.ws, force_general=self.force_general, block_begin=c0, block_count=n)
-            self.ev_done[g].record(main)
-        with torch.cuda.stream(self.s_out):
-            for g, (c0, n) in enumerate(groups):
-                rows = slice(c0 * self.L, (c0 + n) * self.L)
-                self.s_out.wait_event(self.ev_done[g])
-                out_host[rows].copy_(self.out[0, rows], non_blocking=True)
-        main.wait_stream(self.s_out)
+        if (lse_host is None) != (self.lse is None):
+            raise ValueError("lse_host goes with with_lse=True")
+        hp = lambda t: None if t is None else ctypes.c_void_p(t.data_ptr())
+        rc = load().vxl_chunk_prefill_host(
+            hp(q_host), hp(k_host), hp(v_host), self.L, hp(retained_idx_host) if self.R > 0 else None, self.R,
+            hp(out_host), hp(lse_host), _ptr(self.q), _ptr(self.k), _ptr(self.v), _ptr(self.ridx), _ptr(self.out),
+            _ptr(self.lse), self.per_call, ctypes.byref(self.shape), _ptr(self.ws), self.ws.numel(), _stream(stream),
+            ctypes.c_void_p(self.s_in.cuda_stream), ctypes.c_void_p(self.s_out.cuda_stream))
+        if rc != VXL_OK:
+            raise VxlError(rc, "vxl_chunk_prefill_host")
         return out_host
 
 

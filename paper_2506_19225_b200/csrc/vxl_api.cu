@@ -4,6 +4,7 @@
 
 #include <cmath>
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -571,6 +572,119 @@ vxl_status vxl_chunk_prefill_attn(const void *q, const void *k, const void *v, i
     if (!with_prefix) return Cn == 0 ? VXL_OK : launch_prefill_general(p, s, st, false);
 
     return launch_prefill_general(p, s, st);
+}
+
+// Events that order the three streams of vxl_chunk_prefill_host: a pool per device, grown on demand and
+// kept until the process exits.  A wait enqueued on a stream refers to the event's state at that
+// moment, so a later call may record the same events again; the mutex only serialises the enqueueing.
+struct HostPrefillEvents {
+    std::mutex mu;
+    cudaEvent_t *ev = nullptr;
+    int n = 0;
+};
+HostPrefillEvents g_hp_events[kMaxDevices];
+
+bool hp_reserve_events(HostPrefillEvents &pool, int need)
+{
+    if (need <= pool.n) return true;
+    cudaEvent_t *grown = static_cast<cudaEvent_t *>(std::realloc(pool.ev, sizeof(cudaEvent_t) * (size_t)need));
+    if (grown == nullptr) return false;
+    pool.ev = grown;
+    while (pool.n < need) {
+        if (cudaEventCreateWithFlags(&pool.ev[pool.n], cudaEventDisableTiming) != cudaSuccess) return false;
+        ++pool.n;
+    }
+    return true;
+}
+
+vxl_status vxl_chunk_prefill_host(const void *q_host, const void *k_host, const void *v_host, int32_t chunk_len,
+                                  const int32_t *retained_idx_host, int32_t R, void *out_host, float *lse_host,
+                                  void *q_dev, void *k_dev, void *v_dev, int32_t *retained_idx_dev, void *out_dev,
+                                  float *lse_dev, int32_t chunks_per_call, const vxl_shape *s, void *workspace,
+                                  size_t ws_bytes, void *cuda_stream, void *h2d_stream, void *d2h_stream)
+{
+    if (!shape_ok(s) || q_host == nullptr || k_host == nullptr || v_host == nullptr || out_host == nullptr ||
+        q_dev == nullptr || k_dev == nullptr || v_dev == nullptr || out_dev == nullptr)
+        return VXL_ERR_INVALID_ARG;
+    if ((lse_host == nullptr) != (lse_dev == nullptr)) return VXL_ERR_INVALID_ARG;
+    if (chunk_len <= 0 || s->T % chunk_len != 0 || R < 0 || R > chunk_len || chunks_per_call < 0) return VXL_ERR_INVALID_ARG;
+    // plain chunks over back-to-back rows: the host and device arrays share one contiguous layout
+    if (s->prefill_step != 0 && s->prefill_step != chunk_len) return VXL_ERR_UNSUPPORTED;
+    if (s->prefix_len != 0 || s->block_begin != 0 || s->block_count != 0) return VXL_ERR_UNSUPPORTED;
+    const int64_t qrow = (int64_t)s->Hq * s->D, kvrow = (int64_t)s->Hkv * s->D;
+    if (s->q_stride_h != s->D || s->q_stride_t != qrow || s->q_stride_b != (int64_t)s->T * qrow ||
+        s->kv_stride_h != s->D || s->kv_stride_t != kvrow || s->kv_stride_b != (int64_t)s->T * kvrow)
+        return VXL_ERR_UNSUPPORTED;
+    if ((s->out_stride_h != 0 && s->out_stride_h != s->D) || (s->out_stride_t != 0 && s->out_stride_t != qrow) ||
+        (s->out_stride_b != 0 && s->out_stride_b != (int64_t)s->T * qrow))
+        return VXL_ERR_UNSUPPORTED;
+    const int C = s->T / chunk_len;
+    if (R > 0 && C > 1 && (retained_idx_host == nullptr || retained_idx_dev == nullptr)) return VXL_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        ws_bytes < vxl_workspace_bytes(VXL_OP_PREFILL, s, C, R, 0, chunk_len))
+        return VXL_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream), sin = static_cast<cudaStream_t>(h2d_stream),
+                 sout = static_cast<cudaStream_t>(d2h_stream);
+    if (sin == st || sout == st || sin == sout) return VXL_ERR_INVALID_ARG;     // the overlap needs three streams
+
+    const int per = chunks_per_call > 0 ? chunks_per_call : 1;
+    const int groups = (C + per - 1) / per;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VXL_ERR_CUDA;
+    HostPrefillEvents &pool = g_hp_events[dev];
+    std::lock_guard<std::mutex> lock(pool.mu);
+    if (!hp_reserve_events(pool, 2 * groups + 2)) return VXL_ERR_CUDA;
+    cudaEvent_t *ev_in = pool.ev, *ev_done = pool.ev + groups;
+    cudaEvent_t ev_begin = pool.ev[2 * groups], ev_end = pool.ev[2 * groups + 1];
+
+    // the copy streams start after whatever the caller's stream still does with the device arrays
+    if (cudaEventRecord(ev_begin, st) != cudaSuccess || cudaStreamWaitEvent(sin, ev_begin, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(sout, ev_begin, 0) != cudaSuccess)
+        return VXL_ERR_CUDA;
+    if (R > 0 && C > 1 &&
+        cudaMemcpyAsync(retained_idx_dev, retained_idx_host, sizeof(int32_t) * (size_t)C * R, cudaMemcpyHostToDevice, sin) != cudaSuccess)
+        return VXL_ERR_CUDA;
+    const size_t esz = sizeof(__nv_bfloat16), osz = (s->out_dtype == VXL_BF16) ? 2 : 4;
+    // one copy per tensor and chunk group: the rows of the group in every sequence (a 2-D copy whose
+    // pitch is one sequence)
+    auto copy_rows = [&](void *dst, const void *src, int64_t row_elems, size_t elem, int row0, int nrows,
+                         cudaMemcpyKind kind, cudaStream_t cs) {
+        const size_t pitch = (size_t)s->T * row_elems * elem, off = (size_t)row0 * row_elems * elem;
+        return cudaMemcpy2DAsync(static_cast<char *>(dst) + off, pitch, static_cast<const char *>(src) + off, pitch,
+                                 (size_t)nrows * row_elems * elem, (size_t)s->B, kind, cs);
+    };
+    for (int g = 0; g < groups; ++g) {
+        const int c0 = g * per, n = (C - c0 < per) ? C - c0 : per;
+        const int row0 = c0 * chunk_len, nrows = n * chunk_len;
+        if (copy_rows(q_dev, q_host, qrow, esz, row0, nrows, cudaMemcpyHostToDevice, sin) != cudaSuccess ||
+            copy_rows(k_dev, k_host, kvrow, esz, row0, nrows, cudaMemcpyHostToDevice, sin) != cudaSuccess ||
+            copy_rows(v_dev, v_host, kvrow, esz, row0, nrows, cudaMemcpyHostToDevice, sin) != cudaSuccess ||
+            cudaEventRecord(ev_in[g], sin) != cudaSuccess)
+            return VXL_ERR_CUDA;
+    }
+    vxl_shape sub = *s;
+    for (int g = 0; g < groups; ++g) {
+        const int c0 = g * per, n = (C - c0 < per) ? C - c0 : per;
+        if (cudaStreamWaitEvent(st, ev_in[g], 0) != cudaSuccess) return VXL_ERR_CUDA;
+        sub.block_begin = c0; sub.block_count = n;
+        const vxl_status r = vxl_chunk_prefill_attn(q_dev, k_dev, v_dev, chunk_len, retained_idx_dev, R, out_dev, lse_dev, &sub,
+                                                    workspace, ws_bytes, cuda_stream);
+        if (r != VXL_OK) return r;
+        if (cudaEventRecord(ev_done[g], st) != cudaSuccess) return VXL_ERR_CUDA;
+    }
+    for (int g = 0; g < groups; ++g) {
+        const int c0 = g * per, n = (C - c0 < per) ? C - c0 : per;
+        const int row0 = c0 * chunk_len, nrows = n * chunk_len;
+        if (cudaStreamWaitEvent(sout, ev_done[g], 0) != cudaSuccess ||
+            copy_rows(out_host, out_dev, qrow, osz, row0, nrows, cudaMemcpyDeviceToHost, sout) != cudaSuccess)
+            return VXL_ERR_CUDA;
+        if (lse_host != nullptr &&
+            copy_rows(lse_host, lse_dev, s->Hq, sizeof(float), row0, nrows, cudaMemcpyDeviceToHost, sout) != cudaSuccess)
+            return VXL_ERR_CUDA;
+    }
+    // later work on the caller's stream comes after the last copy back
+    if (cudaEventRecord(ev_end, sout) != cudaSuccess || cudaStreamWaitEvent(st, ev_end, 0) != cudaSuccess) return VXL_ERR_CUDA;
+    return VXL_OK;
 }
 
 vxl_status vxl_chunk_scores(const void *q, const void *k_cache, const int32_t *chunk_offsets, int32_t C,

@@ -316,19 +316,30 @@ def test_block_range_with_window_and_prefix():
     check_close(out[0], want, "block range with window and prefix")
 
 
-def test_host_prefill_pipeline_equals_the_oracle_twice_in_a_row():
-    case = inputs.make_prefill(T=2048, L=256, R=32, Hq=4, Hkv=2, D=128, seed=93)
-    hq, hk, hv = (torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory() for x in (case.q, case.k, case.v))
-    hridx = torch.from_numpy(np.ascontiguousarray(case.retained_idx)).pin_memory()
-    hout = torch.empty((case.T, case.Hq, case.D), dtype=torch.float32).pin_memory()
-    hp = vb.HostPrefill(case.T, case.Hq, case.Hkv, case.D, case.L, case.R, chunks_per_call=3, scale=case.scale)
-    want, _ = ref.prefill(case.q, case.k, case.v, case.L, case.retained_idx, case.scale)
+@pytest.mark.parametrize("B,out_dtype,per_call", [(1, torch.float32, 3), (2, torch.bfloat16, 1)])
+def test_host_prefill_pipeline_equals_the_oracle_twice_in_a_row(B, out_dtype, per_call):
+    """vxl_chunk_prefill_host: pinned host q/k/v in, pinned host out (and lse), the pipeline inside the library."""
+    cases = [inputs.make_prefill(T=2048, L=256, R=32, Hq=4, Hkv=2, D=128, seed=93 + b) for b in range(B)]
+    c0 = cases[0]
+    pin = lambda arrs: torch.from_numpy(np.stack([np.ascontiguousarray(a).view(np.int16) for a in arrs])).pin_memory()
+    hq, hk, hv = pin([c.q for c in cases]), pin([c.k for c in cases]), pin([c.v for c in cases])
+    hridx = torch.from_numpy(np.ascontiguousarray(c0.retained_idx)).pin_memory()
+    hout = torch.empty((B, c0.T, c0.Hq, c0.D), dtype=out_dtype).pin_memory()
+    hlse = torch.empty((B, c0.T, c0.Hq), dtype=torch.float32).pin_memory()
+    hp = vb.HostPrefill(c0.T, c0.Hq, c0.Hkv, c0.D, c0.L, c0.R, B=B, chunks_per_call=per_call, scale=c0.scale,
+                        out_dtype=out_dtype, with_lse=True)
+    tol = dict(max_err=2e-2, mean_err=2e-3) if out_dtype == torch.bfloat16 else {}
     for _ in range(2):
-        hout.fill_(float("nan"))
-        hp.run(hq, hk, hv, hridx, hout)
+        hout.fill_(float("nan")); hlse.fill_(float("nan"))
+        hp.run(hq, hk, hv, hridx, hout, hlse)
         torch.cuda.synchronize()
         assert vb.device_status(hp.ws) == vb.VXL_OK
-        check_close(hout, want, "host prefill pipeline")
+        for b, c in enumerate(cases):
+            want, want_lse = ref.prefill(c.q, c.k, c.v, c.L, c0.retained_idx, c.scale)
+            check_close(hout[b].float(), want, f"host prefill pipeline b{b}", **tol)
+            check_close(hlse[b], want_lse, "host prefill lse", max_err=LSE_ABS_ERR, mean_err=LSE_ABS_ERR)
+    # the device arrays hold the sequence afterwards: the KV cache a decoding call would read
+    assert torch.equal(hp.k.cpu().view(torch.int16), hk) and torch.equal(hp.v.cpu().view(torch.int16), hv)
 
 
 def test_ragged_chunks_batched_bf16_out_and_range_fallback():

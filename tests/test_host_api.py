@@ -161,3 +161,32 @@ def test_window_prefix_pool_multi_select_offline_reject_bad_arguments(lib):
     assert o(*args(d, ws_bytes=64)) == vb.VXL_ERR_WORKSPACE
     padded = _shape(B=2, T=512, Hq=28, Hkv=4, D=128, q_strides=(28 * 128, 0, 128), kv_strides=(512 * 640, 640, 128))
     assert o(*args(padded)) == vb.VXL_ERR_UNSUPPORTED               # token rows of the host cache are not contiguous
+
+
+def test_host_prefill_rejects_bad_arguments(lib):
+    """vxl_chunk_prefill_host: refused on the host before any copy or kernel is enqueued."""
+    f = lib.vxl_chunk_prefill_host
+    ws = ctypes.c_void_p(0x20000)
+    s1, s2, s3 = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x2000), ctypes.c_void_p(0x3000)
+    good = _shape(B=1, T=1024, Hq=4, Hkv=2, D=128, q_strides=(1024 * 512, 512, 128), kv_strides=(1024 * 256, 256, 128))
+
+    def call(shape, *, q_host=FAKE, L=256, R=8, lse_host=None, lse_dev=None, ridx_dev=FAKE, per=1, wsb=1 << 30,
+             streams=(s1, s2, s3)):
+        return f(q_host, FAKE, FAKE, L, FAKE, R, FAKE, lse_host, FAKE, FAKE, FAKE, ridx_dev, FAKE, lse_dev, per,
+                 ctypes.byref(shape), ws, wsb, *streams)
+
+    assert call(good, q_host=None) == vb.VXL_ERR_INVALID_ARG
+    assert call(good, L=300) == vb.VXL_ERR_INVALID_ARG                      # T % chunk_len != 0
+    assert call(good, lse_host=FAKE) == vb.VXL_ERR_INVALID_ARG              # lse on one side only
+    assert call(good, ridx_dev=None) == vb.VXL_ERR_INVALID_ARG
+    assert call(good, per=-1) == vb.VXL_ERR_INVALID_ARG
+    assert call(good, wsb=64) == vb.VXL_ERR_WORKSPACE
+    assert call(good, streams=(s1, s1, s3)) == vb.VXL_ERR_INVALID_ARG       # the pipeline needs three streams
+    assert call(good, streams=(s1, s2, s2)) == vb.VXL_ERR_INVALID_ARG
+    padded = _shape(B=1, T=1024, Hq=4, Hkv=2, D=128, q_strides=(1024 * 640, 640, 128), kv_strides=(1024 * 256, 256, 128))
+    assert call(padded) == vb.VXL_ERR_UNSUPPORTED                           # host and device rows are copied whole
+    window = _shape(B=1, T=1024, Hq=4, Hkv=2, D=128, q_strides=(1024 * 512, 512, 128), kv_strides=(1024 * 256, 256, 128), step=128)
+    assert call(window) == vb.VXL_ERR_UNSUPPORTED
+    ranged = _shape(B=1, T=1024, Hq=4, Hkv=2, D=128, q_strides=(1024 * 512, 512, 128), kv_strides=(1024 * 256, 256, 128),
+                    block_begin=1, block_count=1)
+    assert call(ranged) == vb.VXL_ERR_UNSUPPORTED
