@@ -97,9 +97,6 @@ typedef struct vxl_shape {
                                   same buffers.  The prefix rows belong to the call whose range starts at 0 */
     int32_t score_mode;        /* vxl_score_mode, used by vxl_chunk_scores and by
                                   vxl_bilevel_decode_attn when it selects itself              */
-    int32_t decode_split_passes; /* 1: vxl_bilevel_decode_attn always runs its sparse pass, dense pass and
-                                  merge as separate launches; 0: one persistent kernel where the call
-                                  selects itself over a stored sparse level (same results)   */
 } vxl_shape;
 
 /* The sparse level stored on its own (Bi-level KVs Decoding paragraph: both levels of every

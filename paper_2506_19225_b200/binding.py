@@ -36,8 +36,7 @@ class VxlShape(ctypes.Structure):
                 ("scale", ctypes.c_float), ("out_dtype", ctypes.c_int32), ("validate", ctypes.c_int32),
                 ("force_general", ctypes.c_int32), ("prefill_gather4", ctypes.c_int32),
                 ("prefill_step", ctypes.c_int32), ("prefix_len", ctypes.c_int32),
-                ("block_begin", ctypes.c_int32), ("block_count", ctypes.c_int32), ("score_mode", ctypes.c_int32),
-                ("decode_split_passes", ctypes.c_int32)]
+                ("block_begin", ctypes.c_int32), ("block_count", ctypes.c_int32), ("score_mode", ctypes.c_int32)]
 
 
 class VxlSparseLevel(ctypes.Structure):
@@ -133,7 +132,7 @@ def _check_bf16(*ts):
 
 def make_shape(*, B, T, Hq, Hkv, D, q_strides, kv_strides, out_strides=(0, 0, 0), scale=0.0,
                out_dtype=VXL_F32, validate=False, force_general=False, gather4=False, step=0,
-               prefix_len=0, score_mode=VXL_SCORE_LSE, block_begin=0, block_count=0, split_passes=False) -> VxlShape:
+               prefix_len=0, score_mode=VXL_SCORE_LSE, block_begin=0, block_count=0) -> VxlShape:
     s = VxlShape()
     s.struct_size = ctypes.sizeof(VxlShape)
     s.B, s.T, s.Hq, s.Hkv, s.D = B, T, Hq, Hkv, D
@@ -150,7 +149,6 @@ def make_shape(*, B, T, Hq, Hkv, D, q_strides, kv_strides, out_strides=(0, 0, 0)
     s.score_mode = int(score_mode)
     s.block_begin = int(block_begin)
     s.block_count = int(block_count)
-    s.decode_split_passes = int(bool(split_passes))
     return s
 
 
@@ -238,7 +236,7 @@ def prefill_kernel_kind(*, B, T, Hq, Hkv, D, chunk_len, R, force_general=False, 
     return int(load().vxl_prefill_kernel_kind(ctypes.byref(shape), chunk_len, R))
 
 
-def _decode_shape(q, k_cache, out, scale, validate, score_mode=VXL_SCORE_LSE, split_passes=False):
+def _decode_shape(q, k_cache, out, scale, validate, score_mode=VXL_SCORE_LSE):
     B, Hq, D = q.shape
     _, T, Hkv, _ = k_cache.shape
     ostr = (0, 0, 0) if out is None else (out.stride(0), 0, out.stride(1))
@@ -247,7 +245,7 @@ def _decode_shape(q, k_cache, out, scale, validate, score_mode=VXL_SCORE_LSE, sp
                       kv_strides=(k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)),
                       out_strides=ostr, scale=scale or 0.0,
                       out_dtype=VXL_F32 if out is None else _out_code(out.dtype), validate=validate,
-                      score_mode=score_mode, split_passes=split_passes)
+                      score_mode=score_mode)
 
 
 def _ridx_args(retained_idx, C, sparse=None):
@@ -364,10 +362,9 @@ def chunk_scores_static(q, k_cache, chunk_offsets, retained_idx, scores, *, topk
 def bilevel_decode_attn(q, k_cache, v_cache, chunk_offsets, retained_idx, topk: int, *, max_chunk_len: int,
                         selected=None, scale=None, sparse=None, out=None, out_dtype=torch.float32,
                         return_lse=False, return_scores=False, workspace=None, validate=False,
-                        score_mode=VXL_SCORE_LSE, split_passes=False, stream=None):
+                        score_mode=VXL_SCORE_LSE, stream=None):
     """Bi-level KV decoding attention.  Returns a dict with ``out`` [B,Hq,D] and, on request,
-    ``lse`` [B,Hq], ``scores`` [B,C], ``topk`` [B,topk] (only when the call selects itself).
-    ``split_passes`` keeps the sparse pass, the dense pass and the merge as separate launches."""
+    ``lse`` [B,Hq], ``scores`` [B,C], ``topk`` [B,topk] (only when the call selects itself)."""
     _check_bf16(q, k_cache, v_cache)
     if k_cache.stride() != v_cache.stride():
         raise ValueError("k_cache and v_cache must share strides")
@@ -376,7 +373,7 @@ def bilevel_decode_attn(q, k_cache, v_cache, chunk_offsets, retained_idx, topk: 
     ridx, R, rsb = _ridx_args(retained_idx, C, sparse)
     if out is None:
         out = torch.empty((B, Hq, D), dtype=out_dtype, device=q.device)
-    shape = _decode_shape(q, k_cache, out, scale, validate, score_mode, split_passes)
+    shape = _decode_shape(q, k_cache, out, scale, validate, score_mode)
     lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if return_lse else None
     scores = topk_out = None
     if selected is None and return_scores:

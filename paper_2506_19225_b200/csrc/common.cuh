@@ -17,7 +17,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct WsHeader {
     int status;
     int detail;
-    int pad[62];                         // pad[0..3]: grid-wide counters of the one-kernel decode call (zero between calls)
+    int pad[62];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
 

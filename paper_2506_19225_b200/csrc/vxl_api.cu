@@ -14,7 +14,6 @@
 #include "prefill_general.cuh"
 #include "prefill_tc.cuh"
 #include "decode_stream.cuh"
-#include "decode_fused.cuh"
 
 namespace {
 
@@ -35,7 +34,6 @@ bool shape_ok(const vxl_shape *s)
     if (s->Hq % s->Hkv != 0 || s->Hq / s->Hkv > 16) return false;
     if (s->out_dtype != VXL_BF16 && s->out_dtype != VXL_F32) return false;
     if (s->score_mode != VXL_SCORE_LSE && s->score_mode != VXL_SCORE_MASS) return false;
-    if (s->decode_split_passes != 0 && s->decode_split_passes != 1) return false;
     return true;
 }
 
@@ -84,7 +82,7 @@ SlicePlan plan_slices(int B, int topk, int max_chunk_len, int Hkv)
 struct DecodeWs {
     WsHeader *hdr;
     float *part_m, *part_l, *part_o, *score_part;
-    int32_t *sel, *flags, *seq_count;
+    int32_t *sel, *flags;
     size_t bytes;
 };
 
@@ -101,7 +99,6 @@ DecodeWs carve_decode(void *ws, const vxl_shape *s, int C, int topk, int nslices
     w.sel = reinterpret_cast<int32_t *>(base + off); off += align256((size_t)s->B * (topk > 0 ? topk : 1) * sizeof(int32_t));
     w.flags = reinterpret_cast<int32_t *>(base + off); off += align256((size_t)s->B * C * sizeof(int32_t));
     w.score_part = reinterpret_cast<float *>(base + off); off += align256((size_t)s->B * C * s->Hkv * sizeof(float));
-    w.seq_count = reinterpret_cast<int32_t *>(base + off); off += align256((size_t)s->B * sizeof(int32_t));
     w.part_o = reinterpret_cast<float *>(base + off);
     if (with_o) off += align256(nml * s->D * sizeof(float));
     w.bytes = off;
@@ -364,76 +361,6 @@ bool dense_pass_can_select(const vxl_shape *s, const DecodeParams &p, int C, int
     return (int64_t)s->B * topk <= 1024;                     // selections of all sequences fit one CTA's scratch
 }
 
-template <int D, int HPC>
-cudaError_t launch_fused(const FusedMaps &maps, const FusedParams &fp, int grid, cudaStream_t st)
-{
-    static bool done[kMaxDevices] = {};
-    auto kern = decode_fused_kernel<D, HPC>;
-    cudaError_t e = ensure_smem(kern, StreamCfg<D, HPC>::kSmemBytes, done);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(kern, dim3(grid), dim3(StreamCfg<D, HPC>::kThreads), StreamCfg<D, HPC>::kSmemBytes, st, maps, fp);
-}
-
-cudaError_t dispatch_fused(int D, int HPC, const FusedMaps &maps, const FusedParams &fp, int grid, cudaStream_t st)
-{
-    if (D == 128) {
-        if (HPC == 4) return launch_fused<128, 4>(maps, fp, grid, st);
-        if (HPC == 2) return launch_fused<128, 2>(maps, fp, grid, st);
-        return launch_fused<128, 1>(maps, fp, grid, st);
-    }
-    if (HPC == 4) return launch_fused<64, 4>(maps, fp, grid, st);
-    if (HPC == 2) return launch_fused<64, 2>(maps, fp, grid, st);
-    return launch_fused<64, 1>(maps, fp, grid, st);
-}
-
-int device_sm_count()
-{
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    static int sm_count[kMaxDevices] = {};
-    if (dev >= 0 && dev < kMaxDevices) {
-        if (sm_count[dev] == 0) cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
-        if (sm_count[dev] > 0) sms = sm_count[dev];
-    }
-    return sms;
-}
-
-// Scores, selection, both attention passes (and the merge, when one round of merge tasks fits the grid) as
-// one persistent kernel.  *merged = 1 when the output has been written, 0 when the combine kernel must follow.
-cudaError_t run_fused_decode(const vxl_shape *s, const DecodeParams &p, const DecodeWs &w, int C, int topk, void *out,
-                             float *lse, float *scores_out, int32_t *topk_out, int HPC, cudaStream_t st, int *merged)
-{
-    FusedMaps maps;
-    const uint64_t width = (uint64_t)s->Hkv * s->D;
-    const uint32_t box = (uint32_t)stream_tile_rows(HPC);
-    if (!tc_make_map(&maps.ks, p.ks, width, (uint64_t)s->B * C * p.R, width, box) ||
-        !tc_make_map(&maps.vs, p.vs, width, (uint64_t)s->B * C * p.R, width, box) ||
-        !tc_make_map(&maps.k, p.k, width, (uint64_t)s->B * s->T, (uint64_t)s->kv_stride_t, box) ||
-        !tc_make_map(&maps.v, p.v, width, (uint64_t)s->B * s->T, (uint64_t)s->kv_stride_t, box))
-        return cudaErrorUnknown;
-    FusedParams fp;
-    std::memset(&fp, 0, sizeof fp);
-    fp.q = p.q; fp.off = p.off;
-    fp.part_m = w.part_m; fp.part_l = w.part_l; fp.part_o = w.part_o; fp.score_part = w.score_part;
-    fp.sel = w.sel; fp.flags = w.flags; fp.topk_out = topk_out; fp.scores_out = scores_out;
-    fp.seq_count = w.seq_count; fp.sync = reinterpret_cast<int32_t *>(w.hdr) + 2;      // WsHeader::pad fp.hdr = w.hdr;
-    fp.out = out; fp.lse = lse;
-    fp.o_sh = s->out_stride_h ? s->out_stride_h : s->D;
-    fp.o_sb = s->out_stride_b ? s->out_stride_b : (int64_t)s->Hq * fp.o_sh;
-    fp.q_sb = p.q_sb; fp.q_sh = p.q_sh;
-    fp.B = s->B; fp.T = s->T; fp.Hq = s->Hq; fp.Hkv = s->Hkv; fp.G = p.G; fp.C = C; fp.R = p.R; fp.topk = topk;
-    fp.nslices = p.nslices; fp.slice_rows = p.slice_rows; fp.P = p.P; fp.nhb = s->Hkv / HPC;
-    fp.nA = s->B * C * fp.nhb; fp.nB = s->B * topk * p.nslices * fp.nhb;
-    fp.out_bf16 = (s->out_dtype == VXL_BF16);
-    fp.scale_log2 = p.scale_log2;
-    const int sms = device_sm_count();
-    const int64_t items = (int64_t)fp.nA + fp.nB;
-    const int grid = (int)(items < sms ? items : sms);
-    fp.combine = ((int64_t)s->B * s->Hq * (s->D / 32) <= grid) ? 1 : 0;
-    *merged = fp.combine;
-    return dispatch_fused(s->D, HPC, maps, fp, grid, st);
-}
-
 // The passes of one decode call on stream st: (flags from a given selection,) sparse pass, (top-k,)
 // dense pass, combine.  dense_ready: event the dense pass waits for (staged dense rows), or null.
 vxl_status run_decode_passes(const vxl_shape *s, DecodeParams &p, const DecodeWs &w, int C, int R, int topk,
@@ -448,26 +375,16 @@ vxl_status run_decode_passes(const vxl_shape *s, DecodeParams &p, const DecodeWs
         if (cudaGetLastError() != cudaSuccess) return VXL_ERR_CUDA;
         p.flags = w.flags;
     }
-    // One kernel for the whole call where the data layout allows it (stored sparse level, rows of a sequence
-    // back to back, the call picks the chunks itself).
-    const bool fused = selected == nullptr && dense_ready == nullptr && p.staged == 0 && R > 0 && !s->decode_split_passes &&
-                       stream_layout_ok(s) && dense_pass_can_select(s, p, C, topk) &&
-                       (int64_t)s->B * C * (s->Hkv / HPC) + (int64_t)s->B * topk * p.nslices * (s->Hkv / HPC) < (1ll << 30);
-    int merged = 0;
-    if (fused) {
-        if (run_fused_decode(s, p, w, C, topk, out, lse, scores_out, topk_out, HPC, st, &merged) != cudaSuccess) return VXL_ERR_CUDA;
-        if (merged) return VXL_OK;
-    }
-    if (!fused && (R > 0 || selected == nullptr)) {
+    if (R > 0 || selected == nullptr) {
         if (run_sparse_pass<true>(s, p, HPC, st) != cudaSuccess) return VXL_ERR_CUDA;
     }
     // With no selection given, the dense stream pass ranks the chunks itself where it can: one launch fewer.
-    const bool self_select = !fused && selected == nullptr && dense_pass_can_select(s, p, C, topk);
+    const bool self_select = selected == nullptr && dense_pass_can_select(s, p, C, topk);
     if (self_select) {
         p.sel_scores = w.score_part; p.sel_out = w.sel; p.flags_out = w.flags;
         p.topk_out = topk_out; p.scores_out = scores_out;
     }
-    if (!fused && selected == nullptr && !self_select) {
+    if (selected == nullptr && !self_select) {
         if (s->score_mode == VXL_SCORE_MASS) {
             topk_mass_kernel<<<s->B, 1024, (size_t)C * 8, st>>>(tp);
             if (cudaGetLastError() != cudaSuccess) return VXL_ERR_CUDA;
@@ -475,7 +392,7 @@ vxl_status run_decode_passes(const vxl_shape *s, DecodeParams &p, const DecodeWs
             return VXL_ERR_CUDA;
         }
     }
-    if (!fused && topk > 0) {
+    if (topk > 0) {
         p.flags = nullptr;
         if (dense_ready != nullptr && cudaStreamWaitEvent(st, dense_ready, 0) != cudaSuccess) return VXL_ERR_CUDA;
         if (run_dense_pass(s, p, HPC, st) != cudaSuccess) return VXL_ERR_CUDA;

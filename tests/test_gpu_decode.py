@@ -25,13 +25,7 @@ def oracle_selection(d, b, topk, ridx=None):
     return sc, idx, gap
 
 
-def check_decode(d, topk, *, sparse=False, per_seq_ridx=False, split_passes=None):
-    """GPU call against the oracle.  Over a stored sparse level the call is one persistent kernel by default
-    and three launches (sparse pass, dense pass, merge) on request: both are checked."""
-    if split_passes is None:
-        if sparse and d.R > 0:
-            check_decode(d, topk, sparse=sparse, per_seq_ridx=per_seq_ridx, split_passes=True)
-        split_passes = False
+def check_decode(d, topk, *, sparse=False, per_seq_ridx=False):
     q, k, v, off, ridx = gpu_tensors(d)
     ridx_np = d.retained_idx
     if per_seq_ridx:
@@ -41,13 +35,10 @@ def check_decode(d, topk, *, sparse=False, per_seq_ridx=False, split_passes=None
     sp = vb.pack_retained(k, v, ridx) if (sparse and d.R > 0) else None
     ws = vb.new_workspace(vb.workspace_bytes(vb.VXL_OP_DECODE, vb._decode_shape(q, k, None, None, False),
                                              d.C, d.R, topk, d.L), "cuda")
-    res = None
-    for _ in range(2):                       # twice over one workspace: the call leaves its counters at zero
-        res = vb.bilevel_decode_attn(q, k, v, off, ridx, topk, max_chunk_len=d.L, scale=d.scale, sparse=sp,
-                                     return_lse=True, return_scores=True, workspace=ws, validate=True,
-                                     split_passes=split_passes)
-        torch.cuda.synchronize()
-        assert vb.device_status(ws) == vb.VXL_OK
+    res = vb.bilevel_decode_attn(q, k, v, off, ridx, topk, max_chunk_len=d.L, scale=d.scale, sparse=sp,
+                                 return_lse=True, return_scores=True, workspace=ws, validate=True)
+    torch.cuda.synchronize()
+    assert vb.device_status(ws) == vb.VXL_OK
     near_ties = []
     for b in range(d.B):
         rb = ridx_np[b] if per_seq_ridx else ridx_np
@@ -196,10 +187,9 @@ def test_rows_past_the_end_of_an_item_never_reach_the_output():
     k[:, off[C]:] = float("nan"); v[:, off[C]:] = float("nan")             # capacity nobody has written
     off_t, ridx_t = torch.from_numpy(off).cuda(), torch.from_numpy(ridx).cuda()
     level = vb.pack_retained(k, v, ridx_t)
-    for topk, sparse, split in ((2, None, False), (2, level, False), (2, level, True), (C, level, False), (C, level, True),
-                                (1, level, False)):
+    for topk, sparse in ((2, None), (2, level), (C, level), (1, level)):
         res = vb.bilevel_decode_attn(q, k, v, off_t, ridx_t, topk, max_chunk_len=367, scale=d.scale, sparse=sparse,
-                                     return_lse=True, return_scores=True, validate=True, split_passes=split)
+                                     return_lse=True, return_scores=True, validate=True)
         torch.cuda.synchronize()
         assert torch.isfinite(res["out"]).all() and torch.isfinite(res["lse"]).all()
         for b in range(d.B):
@@ -227,13 +217,10 @@ def test_a_selected_chunk_longer_than_max_chunk_len_is_reported():
     level = vb.pack_retained(k, v, ridx)
     shape = vb._decode_shape(q, k, None, None, False)
     ws = vb.new_workspace(vb.workspace_bytes(vb.VXL_OP_DECODE, shape, d.C, d.R, 2, 512), "cuda")
-    for split in (False, True):
-        vb.bilevel_decode_attn(q, k, v, off, ridx, 2, max_chunk_len=256, scale=d.scale, sparse=level, workspace=ws,
-                               split_passes=split)
-        assert vb.device_status(ws) == vb.VXL_ERR_INVALID_ARG          # the bound was not a bound
-        vb.bilevel_decode_attn(q, k, v, off, ridx, 2, max_chunk_len=512, scale=d.scale, sparse=level, workspace=ws,
-                               split_passes=split)
-        assert vb.device_status(ws) == vb.VXL_OK
+    vb.bilevel_decode_attn(q, k, v, off, ridx, 2, max_chunk_len=256, scale=d.scale, sparse=level, workspace=ws)
+    assert vb.device_status(ws) == vb.VXL_ERR_INVALID_ARG              # the bound was not a bound
+    vb.bilevel_decode_attn(q, k, v, off, ridx, 2, max_chunk_len=512, scale=d.scale, sparse=level, workspace=ws)
+    assert vb.device_status(ws) == vb.VXL_OK
 
 
 # ------------------------------------------------------------------ pooled sparse level
@@ -358,7 +345,7 @@ def test_offline_store_decode_matches_oracle_and_the_in_memory_call(B, T, L, R, 
         torch.cuda.synchronize()
         assert vb.device_status(dec.ws) == vb.VXL_OK
         res = vb.bilevel_decode_attn(q, k, v, off, None if pooled else ridx, topk, max_chunk_len=d.L, scale=d.scale,
-                                     sparse=level, return_lse=True, return_scores=True, split_passes=True)
+                                     sparse=level, return_lse=True, return_scores=True)
         assert torch.equal(sel, res["topk"])
         assert (out - res["out"]).abs().max().item() < 1e-5 and (lse - res["lse"]).abs().max().item() < 1e-5
         assert torch.equal(dec.topk_host, sel.cpu())
