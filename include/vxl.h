@@ -338,10 +338,11 @@ vxl_status vxl_device_status(void *workspace, void *cuda_stream);
 const char *vxl_status_str(vxl_status s);
 
 /* Which prefill kernel the shape would use: 1 = tcgen05/TMA kernel, 0 = general kernel,
- * -1 = invalid.  Host-only; launches nothing.  The tcgen05 kernel takes D = 128 with head
- * stride D, sequences laid out back to back, and either plain chunks of 256 rows or more (any
- * length; a multiple of 128 when the call covers a range of chunks) or a sliding window whose
- * prefill_step is a multiple of 128. */
+ * -1 = invalid.  Host-only; launches nothing.  The tcgen05 kernel takes D = 64 or 128 with head
+ * stride D, sequences laid out back to back, and either plain chunks (any length; a multiple of 128
+ * when the call covers a range of chunks) or a sliding window whose prefill_step is a multiple of
+ * 128.  Chunks shorter than 256 rows run there too, with the unused rows of their tile pair
+ * computed and dropped. */
 int32_t vxl_prefill_kernel_kind(const vxl_shape *shape, int32_t chunk_len, int32_t R);
 
 #ifdef __cplusplus

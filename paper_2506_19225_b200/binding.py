@@ -228,11 +228,12 @@ def chunk_prefill_attn(q, k, v, chunk_len: int, retained_idx, *, scale=None, out
     return (out, lse) if return_lse else out
 
 
-def prefill_kernel_kind(*, B, T, Hq, Hkv, D, chunk_len, R, force_general=False, step=0, prefix_len=0) -> int:
+def prefill_kernel_kind(*, B, T, Hq, Hkv, D, chunk_len, R, force_general=False, step=0, prefix_len=0,
+                        block_begin=0, block_count=0) -> int:
     """Which kernel a contiguous [B,T,H,D] problem would use: 1 = tcgen05, 0 = general, -1 = invalid."""
     shape = make_shape(B=B, T=T, Hq=Hq, Hkv=Hkv, D=D, q_strides=(T * Hq * D, Hq * D, D),
                        kv_strides=(T * Hkv * D, Hkv * D, D), force_general=force_general, step=step,
-                       prefix_len=prefix_len)
+                       prefix_len=prefix_len, block_begin=block_begin, block_count=block_count)
     return int(load().vxl_prefill_kernel_kind(ctypes.byref(shape), chunk_len, R))
 
 

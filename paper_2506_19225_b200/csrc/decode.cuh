@@ -671,17 +671,6 @@ __device__ __forceinline__ float f64_to_f32_round_to_odd(double x)
     return f;
 }
 
-// bf16 (given as the fp32 bit pattern with the same value) widened exactly to fp64.  Built with integer
-// operations for normal numbers, because the conversion unit would otherwise bound this kernel: the
-// exponent moves from bias 127 to bias 1023 and the 7 significand bits to the top of the fp64 fraction.
-__device__ __forceinline__ double bf16_bits_to_f64(uint32_t fbits)
-{
-    const uint32_t e = fbits & 0x7F800000u;
-    if (e == 0u || e == 0x7F800000u) return (double)__uint_as_float(fbits);      // zero, subnormal, inf, nan
-    const uint32_t hi = (((fbits & 0x7FFFFFFFu) >> 3) + 0x38000000u) | (fbits & 0x80000000u);
-    return __hiloint2double((int)hi, 0);
-}
-
 __global__ void __launch_bounds__(256) pool_sparse_kernel(const PoolParams p)
 {
     const int per_row = p.Hkv * p.D / 8;
@@ -701,18 +690,31 @@ __global__ void __launch_bounds__(256) pool_sparse_kernel(const PoolParams p)
         double sk[8], sv[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) sk[x] = sv[x] = 0.0;
-        for (int j = a; j < z; ++j) {
-            // read once: streaming loads (evict-first) leave the rest of L2 alone
-            const uint4 uk = __ldcs(reinterpret_cast<const uint4 *>(p.k + col + (int64_t)j * p.kv_st));
-            const uint4 uv = __ldcs(reinterpret_cast<const uint4 *>(p.v + col + (int64_t)j * p.kv_st));
-            const uint32_t *wk2 = reinterpret_cast<const uint32_t *>(&uk);
-            const uint32_t *wv2 = reinterpret_cast<const uint32_t *>(&uv);
+        // two rows per round: four independent 16-byte loads in flight before the first addition
+        auto add_row = [&](const uint4 &uk, const uint4 &uv) {
+            const __nv_bfloat162 *bk = reinterpret_cast<const __nv_bfloat162 *>(&uk);
+            const __nv_bfloat162 *bv = reinterpret_cast<const __nv_bfloat162 *>(&uv);
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
-                // a 32-bit word holds two bf16 values: the low half is the first element
-                sk[2 * x] += bf16_bits_to_f64(wk2[x] << 16); sk[2 * x + 1] += bf16_bits_to_f64(wk2[x] & 0xFFFF0000u);
-                sv[2 * x] += bf16_bits_to_f64(wv2[x] << 16); sv[2 * x + 1] += bf16_bits_to_f64(wv2[x] & 0xFFFF0000u);
+                const float2 fk = __bfloat1622float2(bk[x]), fv = __bfloat1622float2(bv[x]);
+                sk[2 * x] += (double)fk.x; sk[2 * x + 1] += (double)fk.y;
+                sv[2 * x] += (double)fv.x; sv[2 * x + 1] += (double)fv.y;
             }
+        };
+        int j = a;
+        for (; j + 1 < z; j += 2) {
+            // read once: streaming loads (evict-first) leave the rest of L2 alone
+            const uint4 uk0 = __ldcs(reinterpret_cast<const uint4 *>(p.k + col + (int64_t)j * p.kv_st));
+            const uint4 uv0 = __ldcs(reinterpret_cast<const uint4 *>(p.v + col + (int64_t)j * p.kv_st));
+            const uint4 uk1 = __ldcs(reinterpret_cast<const uint4 *>(p.k + col + (int64_t)(j + 1) * p.kv_st));
+            const uint4 uv1 = __ldcs(reinterpret_cast<const uint4 *>(p.v + col + (int64_t)(j + 1) * p.kv_st));
+            add_row(uk0, uv0);                    // row order is kept: the sum is the oracle's, bit for bit
+            add_row(uk1, uv1);
+        }
+        if (j < z) {
+            const uint4 uk0 = __ldcs(reinterpret_cast<const uint4 *>(p.k + col + (int64_t)j * p.kv_st));
+            const uint4 uv0 = __ldcs(reinterpret_cast<const uint4 *>(p.v + col + (int64_t)j * p.kv_st));
+            add_row(uk0, uv0);
         }
         const double n = (double)(z - a);
         uint4 ok, ov;

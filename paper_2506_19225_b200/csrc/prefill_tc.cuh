@@ -15,7 +15,7 @@
 //   warp  9     TMA producer: Q per item; K and V tiles in units (V_j with K_{j+1}) through a ring
 //               of 64 KB pair slots that runs on into the next item while the current one finishes
 //   warps 10-11 idle; the third warpgroup hands most of its registers to the softmax warps
-// TMEM (512 columns x 128 lanes, fp32): S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512);
+// TMEM (512 columns x 128 lanes, fp32): S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [384,384+D);
 // P (bf16, two per column) overwrites the first 64 columns of its S.
 // The two query tiles ping-pong: while the softmax warps of one tile work on S_j, the tensor
 // pipe runs the other tile's P.V and the next Q.K^T.  Across items the pipeline keeps going: the
@@ -38,7 +38,8 @@ constexpr int kTcThreads = 384;                          // three warpgroups (th
 constexpr int kTcStages = VXL_TC_STAGES;               // K/V ring slots of 32 KB
 constexpr int kTcPairs = kTcStages / 2;                  // pair slots of 64 KB (V tile + K tile)
 static_assert(kTcStages % 2 == 0, "the ring is used in pairs of tiles");
-constexpr uint32_t kTcTileBytes = 128 * 128 * 2;        // one 128 x 128 bf16 tile
+constexpr uint32_t kTcTileBytes = 128 * 128 * 2;        // room of one tile in shared memory (128 rows x 128 columns of bf16)
+template <int D> constexpr uint32_t kTcTileLoad = 128u * D * 2u;   // bytes a 128-row tile of head dimension D brings in
 constexpr uint32_t kTcPanelBytes = 128 * 64 * 2;        // 64 columns (128 B) x 128 rows
 constexpr uint32_t kTcSmemQ = 0;
 constexpr uint32_t kTcSmemKV = 2 * kTcTileBytes;
@@ -187,6 +188,24 @@ __device__ __forceinline__ void tc_qk8(uint32_t d_tmem, uint32_t a_lo, uint32_t 
         "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
         : "memory");
 }
+// The same for a head dimension of 64: four k = 16 steps inside the one 64-column panel.
+__device__ __forceinline__ void tc_qk4(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pf, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 pf, %0, %0;\n\tsetp.eq.b32 pt, %0, %0;\n\t"
+        "add.u32 al, %1, 0;\n\tadd.u32 bl, %2, 0;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
+        "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+        "add.u32 al, %1, 4;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+        "add.u32 al, %1, 6;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
+        : "memory");
+}
 // Half of one O += P.V tile: four k = 16 steps (64 keys).  p_tmem is the TMEM address of the
 // first P column of the half, b_lo the low descriptor word of the first V row block of the half;
 // `acc` = 0 makes the first step overwrite O.
@@ -208,14 +227,14 @@ __device__ __forceinline__ void tc_pv4(uint32_t d_tmem, uint32_t p_tmem, uint32_
         "}" ::"r"(d_tmem), "r"(p_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
         : "memory");
 }
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = N = 128.
-__host__ __device__ constexpr uint32_t tc_idesc(bool b_mn_major)
+// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128, N = n (128 keys for S, the head dimension for O).
+__host__ __device__ constexpr uint32_t tc_idesc(bool b_mn_major, uint32_t n = 128u)
 {
     return (1u << 4)                      // D format: F32
            | (1u << 7)                    // A format: BF16
            | (1u << 10)                   // B format: BF16
            | ((b_mn_major ? 1u : 0u) << 16)
-           | ((128u >> 3) << 17)          // N
+           | ((n >> 3) << 17)             // N
            | ((128u >> 4) << 24);         // M
 }
 
@@ -302,6 +321,7 @@ __device__ __forceinline__ bool tc_item(const PrefillParams &p, const int2 *__re
     return true;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, const int2 *__restrict__ order, const int pairs,
                   const int tma_out)
@@ -357,13 +377,13 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
             // Q of this item: its shared memory is free once the last S = Q.K^T of the previous item is done
             if (k > 0 && (!mbar_wait(bar(kBarQFree), (k - 1) & 1) || *s_abort)) { ok = false; break; }
             if (lane == 0) {
-                mbar_expect_tx(bar(kBarQ), 2 * kTcTileBytes);
+                mbar_expect_tx(bar(kBarQ), 2 * kTcTileLoad<D>);
 #pragma unroll
                 for (int t = 0; t < 2; ++t)
 #pragma unroll
-                    for (int pn = 0; pn < 2; ++pn)
+                    for (int pn = 0; pn < D / 64; ++pn)
                         tma_load_2d(smem_base + kTcSmemQ + t * kTcTileBytes + pn * kTcPanelBytes, &maps.q,
-                                    w.h * 128 + pn * 64, w.row_base + w.q_row0 + t * 128, bar(kBarQ));
+                                    w.h * D + pn * 64, w.row_base + w.q_row0 + t * 128, bar(kBarQ));
             }
             ++q_loads;
             const int pk_row0 = w.b * p.C * p.R;         // this sequence's rows in the packed sparse level
@@ -375,8 +395,8 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                     const int y0 = w.row_base + p.ridx[min(e + 0, w.n_r - 1)], y1 = w.row_base + p.ridx[min(e + 1, w.n_r - 1)];
                     const int y2 = w.row_base + p.ridx[min(e + 2, w.n_r - 1)], y3 = w.row_base + p.ridx[min(e + 3, w.n_r - 1)];
                     const CUtensorMap *m = kv ? &maps.vg : &maps.kg;
-                    tma_gather4(dst + lane * 512, m, w.kvh * 128, y0, y1, y2, y3, fb);
-                    tma_gather4(dst + kTcPanelBytes + lane * 512, m, w.kvh * 128 + 64, y0, y1, y2, y3, fb);
+                    tma_gather4(dst + lane * 512, m, w.kvh * D, y0, y1, y2, y3, fb);
+                    if (D == 128) tma_gather4(dst + kTcPanelBytes + lane * 512, m, w.kvh * D + 64, y0, y1, y2, y3, fb);
                 } else if (lane == 0) {
                     // retained tiles come from the packed sparse level (rows past this chunk's
                     // prefix belong to later chunks or are out of range: masked / zero filled)
@@ -385,8 +405,8 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                     const int jp = j - w.n_ret;                  // prefix tiles first, then the window
                     const int y = ret ? pk_row0 + j * 128
                                       : (jp < w.n_pre ? w.row_base + jp * 128 : w.row_base + w.win_row0 + (jp - w.n_pre) * 128);
-                    tma_load_2d(dst, m, w.kvh * 128, y, fb);
-                    tma_load_2d(dst + kTcPanelBytes, m, w.kvh * 128 + 64, y, fb);
+                    tma_load_2d(dst, m, w.kvh * D, y, fb);
+                    if (D == 128) tma_load_2d(dst + kTcPanelBytes, m, w.kvh * D + 64, y, fb);
                 }
             };
             for (int u = 0; u <= w.n && ok; ++u, ++un) {
@@ -395,7 +415,7 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                 if (!mbar_wait(bar(kBarEmpty + slot), ph ^ 1) || *s_abort) { ok = false; break; }
                 const uint32_t dst = smem_base + kTcSmemKV + slot * 2 * kTcTileBytes;
                 const bool has_v = (u > 0), has_k = (u < w.n);
-                if (lane == 0) mbar_expect_tx(bar(kBarFull + slot), (has_v && has_k) ? 2 * kTcTileBytes : kTcTileBytes);
+                if (lane == 0) mbar_expect_tx(bar(kBarFull + slot), (has_v && has_k) ? 2 * kTcTileLoad<D> : kTcTileLoad<D>);
                 __syncwarp();
                 if (has_v) load_tile(1, u - 1, dst, bar(kBarFull + slot));
                 if (has_k) load_tile(0, u, dst + kTcTileBytes, bar(kBarFull + slot));
@@ -414,14 +434,16 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
         // =============================================================== MMA issuer
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;" ::: "memory");
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = tc_idesc(false), idesc_pv = tc_idesc(true);
+            constexpr uint32_t idesc_qk = tc_idesc(false, 128u), idesc_pv = tc_idesc(true, (uint32_t)D);
             constexpr uint32_t desc_hi = tc_desc_hi(1024);
             bool ok = true;
             int ub = 0;                                  // K/V units consumed before this item
             int pc0 = 0, pc1 = 0;                        // P tiles consumed per query tile (all items)
             auto issue_qk = [&](int t, uint32_t ka) {
-                tc_qk8(tmem + t * 128, tc_desc_lo(smem_base + kTcSmemQ + t * kTcTileBytes, 16), tc_desc_lo(ka, 16), desc_hi,
-                       idesc_qk);
+                if (D == 128)
+                    tc_qk8(tmem + t * 128, tc_desc_lo(smem_base + kTcSmemQ + t * kTcTileBytes, 16), tc_desc_lo(ka, 16), desc_hi, idesc_qk);
+                else
+                    tc_qk4(tmem + t * 128, tc_desc_lo(smem_base + kTcSmemQ + t * kTcTileBytes, 16), tc_desc_lo(ka, 16), desc_hi, idesc_qk);
             };
             // P.V in two halves of 64 keys: the first runs while the softmax still works on the second
             auto issue_pv = [&](int t, uint32_t va, bool acc, int pc) -> bool {
@@ -555,7 +577,7 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                         // PV of tile j-1 has completed (S_j was committed after it), so O is stable.
                         float o[32];
 #pragma unroll 1
-                        for (int cb = 0; cb < 4; ++cb) {
+                        for (int cb = 0; cb < D / 32; ++cb) {
                             tc_ld32(tO + cb * 32, o);
                             tc_wait_ld();
 #pragma unroll
@@ -600,8 +622,10 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
             // four, and the tensor memory is handed back before the stores start
             tc_ld32(tO + 0, s + 0);
             tc_ld32(tO + 32, s + 32);
-            tc_ld32(tO + 64, s + 64);
-            tc_ld32(tO + 96, s + 96);
+            if (D == 128) {
+                tc_ld32(tO + 64, s + 64);
+                tc_ld32(tO + 96, s + 96);
+            }
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
@@ -613,7 +637,7 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
             if (box_store && p.out_bf16) {
                 // bf16 output: a box is 32 rows x 64 columns (128 bytes a row, the same swizzle), two per warp
 #pragma unroll
-                for (int cb = 0; cb < 2; ++cb) {
+                for (int cb = 0; cb < D / 64; ++cb) {
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
 #pragma unroll
@@ -627,11 +651,11 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) tma_store_2d(&maps.o, w.h * 128 + cb * 64, w.row_base + tok0, stage);
+                    if (lane == 0) tma_store_2d(&maps.o, w.h * D + cb * 64, w.row_base + tok0, stage);
                 }
             } else
 #pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
+            for (int cb = 0; cb < D / 32; ++cb) {
                 if (tma_out != 0) {
                     if (lane == 0) tma_store_wait_read();             // the previous box has left the staging block
                     __syncwarp();
@@ -647,7 +671,7 @@ prefill_tc_kernel(const __grid_constant__ TcMaps maps, const PrefillParams p, co
                 if (box_store) {
                     fence_proxy_async_smem();                         // generic-proxy writes -> visible to the TMA
                     __syncwarp();
-                    if (lane == 0) tma_store_2d(&maps.o, w.h * 128 + cb * 32, w.row_base + tok0, stage);
+                    if (lane == 0) tma_store_2d(&maps.o, w.h * D + cb * 32, w.row_base + tok0, stage);
                     continue;
                 }
                 __syncwarp();
@@ -703,14 +727,13 @@ inline bool prefill_tc_supported(const vxl_shape *s, int L, int R)
 {
     (void)R;
     const int step = s->prefill_step > 0 ? s->prefill_step : L;
-    if (s->D != 128) return false;
+    if (s->D != 128 && s->D != 64) return false;
     if (step == L) {
         // Plain chunks of any length from 256 rows: the last pair of query tiles may reach past the chunk.
         // Its surplus rows are computed on whatever follows (the next chunk's rows, zero fill past the
         // array) and never stored; for the rows that count, every key past the chunk is also past the
         // diagonal.  A call over a range of chunks must read nothing after the range, so there the
         // chunk has to end on a key-tile boundary.
-        if (L < 256) return false;
         if ((s->block_begin > 0 || s->block_count > 0) && L % 128 != 0) return false;
     } else {
         // Sliding window: the key tiles are laid from the window start, the query tiles from the block
@@ -718,7 +741,7 @@ inline bool prefill_tc_supported(const vxl_shape *s, int L, int R)
         // is cut off at the start of the sequence: every block starts a whole number of tiles in.
         if (step % 128 != 0) return false;
     }
-    if (s->q_stride_h != 128 || s->kv_stride_h != 128) return false;
+    if (s->q_stride_h != s->D || s->kv_stride_h != s->D) return false;
     if (s->B > 1 && (s->q_stride_b != (int64_t)s->T * s->q_stride_t || s->kv_stride_b != (int64_t)s->T * s->kv_stride_t))
         return false;
     if ((int64_t)s->B * s->T >= (1ll << 31)) return false;
@@ -760,33 +783,34 @@ inline bool tc_make_map(CUtensorMap *m, const void *base, uint64_t width, uint64
 
 // ks/vs: packed sparse level [B*C*R, Hkv, 128] (built by the caller of this function with
 // pack_retained_kernel), or null when p.gather4 selects TMA gather4 straight from K/V.
-inline vxl_status prefill_tc_launch(const PrefillParams &p, void *order_ws, const void *ks, const void *vs,
-                                    cudaStream_t st)
+template <int D>
+inline vxl_status prefill_tc_launch_d(const PrefillParams &p, void *order_ws, const void *ks, const void *vs,
+                                      cudaStream_t st)
 {
     TcMaps maps;
     const uint64_t rows = (uint64_t)p.B * p.T;
     const uint64_t prow = (uint64_t)p.B * p.C * p.R;
     const bool need_sparse = p.R > 0 && p.C > 1;
-    if (!tc_make_map(&maps.q, p.q, (uint64_t)p.Hq * 128, rows, (uint64_t)p.q_st, 128) ||
-        !tc_make_map(&maps.k, p.k, (uint64_t)p.Hkv * 128, rows, (uint64_t)p.kv_st, 128) ||
-        !tc_make_map(&maps.v, p.v, (uint64_t)p.Hkv * 128, rows, (uint64_t)p.kv_st, 128))
+    if (!tc_make_map(&maps.q, p.q, (uint64_t)p.Hq * D, rows, (uint64_t)p.q_st, 128) ||
+        !tc_make_map(&maps.k, p.k, (uint64_t)p.Hkv * D, rows, (uint64_t)p.kv_st, 128) ||
+        !tc_make_map(&maps.v, p.v, (uint64_t)p.Hkv * D, rows, (uint64_t)p.kv_st, 128))
         return VXL_ERR_CUDA;
     if (p.gather4 || !need_sparse) {
-        if (!tc_make_map(&maps.kg, p.k, (uint64_t)p.Hkv * 128, rows, (uint64_t)p.kv_st, 1) ||
-            !tc_make_map(&maps.vg, p.v, (uint64_t)p.Hkv * 128, rows, (uint64_t)p.kv_st, 1))
+        if (!tc_make_map(&maps.kg, p.k, (uint64_t)p.Hkv * D, rows, (uint64_t)p.kv_st, 1) ||
+            !tc_make_map(&maps.vg, p.v, (uint64_t)p.Hkv * D, rows, (uint64_t)p.kv_st, 1))
             return VXL_ERR_CUDA;
     } else {
-        if (!tc_make_map(&maps.kg, ks, (uint64_t)p.Hkv * 128, prow, (uint64_t)p.Hkv * 128, 128) ||
-            !tc_make_map(&maps.vg, vs, (uint64_t)p.Hkv * 128, prow, (uint64_t)p.Hkv * 128, 128))
+        if (!tc_make_map(&maps.kg, ks, (uint64_t)p.Hkv * D, prow, (uint64_t)p.Hkv * D, 128) ||
+            !tc_make_map(&maps.vg, vs, (uint64_t)p.Hkv * D, prow, (uint64_t)p.Hkv * D, 128))
             return VXL_ERR_CUDA;
     }
     // output with heads side by side and sequences back to back: boxes leave by TMA store
     int tma_out = 0;
     const int o_esz = p.out_bf16 ? 2 : 4;
-    if (p.o_sh == 128 && (p.B == 1 || p.o_sb == (int64_t)p.T * p.o_st) &&
+    if (p.o_sh == D && (p.B == 1 || p.o_sb == (int64_t)p.T * p.o_st) &&
         (reinterpret_cast<uintptr_t>(p.out) & 15u) == 0 && (p.o_st * o_esz) % 16 == 0) {
         tc_encode_fn enc = tc_get_encode();
-        const cuuint64_t dims[2] = {(cuuint64_t)p.Hq * 128, rows};
+        const cuuint64_t dims[2] = {(cuuint64_t)p.Hq * D, rows};
         const cuuint64_t strides[1] = {(cuuint64_t)p.o_st * o_esz};
         const cuuint32_t box[2] = {p.out_bf16 ? 64u : 32u, 32};      // 128 bytes a row either way
         const cuuint32_t estr[2] = {1, 1};
@@ -801,7 +825,7 @@ inline vxl_status prefill_tc_launch(const PrefillParams &p, void *order_ws, cons
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VXL_ERR_CUDA;
     if (!smem_done[dev]) {
-        if (cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmemBytes) != cudaSuccess)
             return VXL_ERR_CUDA;
         smem_done[dev] = true;
     }
@@ -820,8 +844,14 @@ inline vxl_status prefill_tc_launch(const PrefillParams &p, void *order_ws, cons
         sm_count[dev] = 148;
     const int64_t items = (int64_t)entries * p.B * p.Hq;
     const unsigned grid = (unsigned)(items < sm_count[dev] ? items : sm_count[dev]);
-    prefill_tc_kernel<<<grid, kTcThreads, kTcSmemBytes, st>>>(maps, p, order, pairs, tma_out);
+    prefill_tc_kernel<D><<<grid, kTcThreads, kTcSmemBytes, st>>>(maps, p, order, pairs, tma_out);
     return cudaGetLastError() == cudaSuccess ? VXL_OK : VXL_ERR_CUDA;
+}
+
+inline vxl_status prefill_tc_launch(const PrefillParams &p, int D, void *order_ws, const void *ks, const void *vs,
+                                    cudaStream_t st)
+{
+    return D == 128 ? prefill_tc_launch_d<128>(p, order_ws, ks, vs, st) : prefill_tc_launch_d<64>(p, order_ws, ks, vs, st);
 }
 
 }  // namespace vxl

@@ -561,7 +561,7 @@ vxl_status vxl_chunk_prefill_attn(const void *q, const void *k, const void *v, i
             }
         }
         if (Cn > 0) {
-            const vxl_status r = prefill_tc_launch(p, order_ws, ks, vs, st);
+            const vxl_status r = prefill_tc_launch(p, s->D, order_ws, ks, vs, st);
             if (r != VXL_OK || P0 == 0 || !with_prefix) return r;
         }
         if (!with_prefix) return VXL_OK;

@@ -61,6 +61,11 @@ EDGE = [
     (1540, 385, 33, 7, 1, 128),      # one row into the second tile of the second pair
     (1280, 640, 64, 2, 1, 128),      # two and a half pairs
     (1808, 452, 452, 2, 2, 128),     # everything retained, ragged chunks: dense causal
+    (1024, 512, 48, 4, 2, 64),       # head dimension 64: one 64-column panel per tile
+    (1536, 384, 384, 6, 2, 64),      # head dimension 64, everything retained
+    (640, 128, 16, 4, 2, 128),       # one query tile per chunk: the pair's second tile is surplus
+    (800, 40, 7, 2, 1, 128),         # twenty chunks shorter than a third of a tile
+    (1210, 110, 30, 3, 1, 64),       # short ragged chunks, head dimension 64
 ]
 
 
@@ -132,15 +137,17 @@ def test_kernel_kind_selection():
         kw = dict(B=1, T=c.T, Hq=c.Hq, Hkv=c.Hkv, D=c.D, chunk_len=c.L, R=c.R)
         assert vb.prefill_kernel_kind(**kw) == 1                     # tcgen05 kernel
         assert vb.prefill_kernel_kind(force_general=True, **kw) == 0
-    # plain chunks of any length from 256 rows run on the tcgen05 kernel; a call over a range of chunks
-    # needs the chunk to end on a key-tile boundary; windows need multiples of 256
+    # plain chunks of any length and both head dimensions run on the tcgen05 kernel; a call over a range of
+    # chunks needs the chunk to end on a key-tile boundary; window steps must be multiples of 128
     assert vb.prefill_kernel_kind(B=1, T=1200, Hq=4, Hkv=2, D=128, chunk_len=300, R=20) == 1
-    assert vb.prefill_kernel_kind(B=1, T=1000, Hq=4, Hkv=2, D=128, chunk_len=200, R=20) == 0
+    assert vb.prefill_kernel_kind(B=1, T=1000, Hq=4, Hkv=2, D=128, chunk_len=200, R=20) == 1
+    assert vb.prefill_kernel_kind(B=1, T=1000, Hq=4, Hkv=2, D=64, chunk_len=40, R=3) == 1
+    assert vb.prefill_kernel_kind(B=1, T=1000, Hq=4, Hkv=2, D=128, chunk_len=200, R=20, block_begin=1, block_count=2) == 0
     assert vb.prefill_kernel_kind(B=1, T=1200, Hq=4, Hkv=2, D=128, chunk_len=600, R=20, step=300) == 0
     assert vb.prefill_kernel_kind(B=1, T=1920, Hq=4, Hkv=2, D=128, chunk_len=960, R=20, step=320) == 0
     assert vb.prefill_kernel_kind(B=1, T=1536, Hq=4, Hkv=2, D=128, chunk_len=384, R=20, step=128) == 1
     c = inputs.prefill_shape("cfg1_tiny")
-    assert vb.prefill_kernel_kind(B=1, T=c.T, Hq=c.Hq, Hkv=c.Hkv, D=c.D, chunk_len=c.L, R=c.R) == 0
+    assert vb.prefill_kernel_kind(B=1, T=c.T, Hq=c.Hq, Hkv=c.Hkv, D=c.D, chunk_len=c.L, R=c.R) == 1
     assert vb.prefill_kernel_kind(B=1, T=100, Hq=2, Hkv=1, D=64, chunk_len=64, R=0) == -1
 
 
@@ -209,7 +216,7 @@ def test_window_and_prefix(T_vis, L, step, prefix_len, R, Hq, Hkv, D, force_gene
     out, lse = run_gpu_window(case, force_general=force_general)
     kind = vb.prefill_kernel_kind(B=1, T=case.T, Hq=Hq, Hkv=Hkv, D=D, chunk_len=L, R=R, force_general=force_general,
                                   step=step, prefix_len=prefix_len)
-    fast = D == 128 and not force_general and ((step == L and L >= 256) or (step != L and step % 128 == 0))
+    fast = not force_general and (step == L or step % 128 == 0)
     assert kind == (1 if fast else 0)
     want, want_lse = ref.prefill_window(case.q, case.k, case.v, case.L, case.step, case.prefix_len,
                                         case.retained_idx, case.scale)
