@@ -120,9 +120,32 @@ __global__ void __launch_bounds__(32 * (kDecWarps + 1)) decode_partial_kernel(co
         // ------------------------------------------------------------ producer
         int issued = 0;
         const uint64_t row_policy = l2_evict_first_policy();        // every row is read once per call
+        // Rows fetched by index: the positions of a tile are read from retained_idx one tile ahead, so that
+        // the load's round trip runs under the wait for a free stage and the copies of the tile before.
+        constexpr int RPL = (TK + 31) / 32;                          // rows per lane and tile
+        const bool by_index = SPARSE && !packed;
+        int64_t pos_next[RPL];
+        auto fetch_pos = [&](int it2) {
+#pragma unroll
+            for (int i = 0; i < RPL; ++i) pos_next[i] = 0;
+            if (!by_index || it2 >= ntiles) return;
+            const int r0 = tile_row0(it2);
+            const int nv = min(TK, len - r0);
+            if (nv <= 0) return;
+#pragma unroll
+            for (int i = 0; i < RPL; ++i) {
+                const int r = lane + 32 * i;
+                if (r < TK) pos_next[i] = p.ridx[(int64_t)b * p.ridx_sb + (int64_t)chunk * p.R + r0 + min(r, nv - 1)];
+            }
+        };
+        fetch_pos(0);
         for (int it = 0; it < ntiles; ++it) {
             const int row0 = tile_row0(it);
             const int nvalid = min(TK, len - row0);
+            int64_t pos_cur[RPL];
+#pragma unroll
+            for (int i = 0; i < RPL; ++i) pos_cur[i] = pos_next[i];
+            fetch_pos(it + 1);
             if (nvalid <= 0) continue;
             const int stage = issued % kDecStages;
             const uint32_t ph = (issued / kDecStages) & 1;
@@ -135,7 +158,10 @@ __global__ void __launch_bounds__(32 * (kDecWarps + 1)) decode_partial_kernel(co
             __syncwarp();
             __nv_bfloat16 *dK = ring + (size_t)stage * 2 * Cfg::TILE;
             __nv_bfloat16 *dV = dK + Cfg::TILE;
-            for (int r = lane; r < TK; r += 32) {
+#pragma unroll
+            for (int ri = 0; ri < RPL; ++ri) {
+                const int r = lane + 32 * ri;
+                if (r >= TK) break;
                 const int rr = min(r, nvalid - 1);                  // tail rows repeat a valid row (masked later)
                 const __nv_bfloat16 *srcK, *srcV;
                 int64_t hstride;
@@ -146,7 +172,7 @@ __global__ void __launch_bounds__(32 * (kDecWarps + 1)) decode_partial_kernel(co
                         srcV = WITH_V ? p.vs + (e * p.Hkv + (int64_t)hb * HPC) * D : nullptr;
                         hstride = D;
                     } else {
-                        int64_t pos = p.ridx[(int64_t)b * p.ridx_sb + (int64_t)chunk * p.R + row0 + rr];
+                        int64_t pos = pos_cur[ri];
                         pos = pos < 0 ? 0 : (pos >= p.T ? p.T - 1 : pos);
                         const int64_t o = kv_b + pos * p.kv_st + (int64_t)hb * HPC * p.kv_sh;
                         srcK = p.k + o; srcV = WITH_V ? p.v + o : nullptr; hstride = p.kv_sh;

@@ -270,17 +270,19 @@ __device__ __forceinline__ int tc_entry_cost(int c, int pr, int R, int S, int L)
 }
 __global__ void __launch_bounds__(1024) prefill_tc_order_kernel(int2 *order, int c0, int Cn, int pairs, int R, int S, int L)
 {
+    __shared__ int s_cost[kTcMaxOrder];
     const int n = Cn * pairs;                             // blocks c0 .. c0 + Cn - 1
+    for (int e = threadIdx.x; e < n; e += blockDim.x) s_cost[e] = tc_entry_cost(c0 + e / pairs, e % pairs, R, S, L);
+    __syncthreads();
     for (int e = threadIdx.x; e < n; e += blockDim.x) {
-        const int c = c0 + e / pairs, pr = e % pairs;
-        const int cost = tc_entry_cost(c, pr, R, S, L);
+        const int cost = s_cost[e];
         int rank = 0;
+#pragma unroll 8
         for (int e2 = 0; e2 < n; ++e2) {
-            const int c2 = c0 + e2 / pairs, p2 = e2 % pairs;
-            const int cost2 = tc_entry_cost(c2, p2, R, S, L);
+            const int cost2 = s_cost[e2];
             rank += (cost2 > cost || (cost2 == cost && e2 < e)) ? 1 : 0;
         }
-        order[rank] = make_int2(c, pr);
+        order[rank] = make_int2(c0 + e / pairs, e % pairs);
     }
 }
 
