@@ -334,6 +334,14 @@ vxl_status vxl_pool_sparse(const void *k_cache, const void *v_cache,
  * the device-side error recorded since the last clear, or VXL_ERR_CUDA. */
 vxl_status vxl_device_status(void *workspace, void *cuda_stream);
 
+/* Self-test of the failure path every kernel of this library shares (the paper has no counterpart).  All
+ * device-side waits are bounded: when one runs out, the kernel records VXL_ERR_TIMEOUT in the workspace's
+ * status word and returns, and the context stays usable.  This call launches one warp that waits, with that
+ * same bounded wait and a limit of limit_cycles SM clocks (1 .. 200,000,000), on a barrier that nothing
+ * completes; vxl_device_status(workspace) must then report VXL_ERR_TIMEOUT, and the next call on the same
+ * workspace must work.  workspace: at least 256 bytes, 256-byte aligned, device memory. */
+vxl_status vxl_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream);
+
 /* Static, NUL-terminated description of a status code (host memory, never freed). */
 const char *vxl_status_str(vxl_status s);
 

@@ -23,7 +23,7 @@ VXL_OP_PREFILL, VXL_OP_SCORES, VXL_OP_DECODE = 0, 1, 2
 VXL_SCORE_LSE, VXL_SCORE_MASS = 0, 1
 
 EXPORTS = ("vxl_workspace_bytes", "vxl_chunk_prefill_attn", "vxl_chunk_prefill_host", "vxl_chunk_scores",
-           "vxl_chunk_scores_static", "vxl_chunk_scores_multi", "vxl_topk_select", "vxl_bilevel_decode_attn", "vxl_bilevel_decode_offline", "vxl_pack_retained", "vxl_pool_sparse", "vxl_device_status",
+           "vxl_chunk_scores_static", "vxl_chunk_scores_multi", "vxl_topk_select", "vxl_bilevel_decode_attn", "vxl_bilevel_decode_offline", "vxl_pack_retained", "vxl_pool_sparse", "vxl_device_status", "vxl_selftest_bounded_wait",
            "vxl_status_str", "vxl_prefill_kernel_kind")
 
 
@@ -99,6 +99,8 @@ def load():
         lib.vxl_pool_sparse.argtypes = [vp, vp, vp, i32, i32, vp, vp, ctypes.POINTER(VxlShape), vp]
         lib.vxl_device_status.restype = ctypes.c_int
         lib.vxl_device_status.argtypes = [vp, vp]
+        lib.vxl_selftest_bounded_wait.restype = ctypes.c_int
+        lib.vxl_selftest_bounded_wait.argtypes = [vp, i64, vp]
         _lib = lib
     return _lib
 
@@ -163,6 +165,11 @@ def new_workspace(nbytes: int, device) -> torch.Tensor:
 
 def device_status(workspace: torch.Tensor, stream=None) -> int:
     return int(load().vxl_device_status(_ptr(workspace), _stream(stream)))
+
+
+def selftest_bounded_wait(workspace: torch.Tensor, limit_cycles: int = 2_000_000, stream=None) -> int:
+    """Launches the probe whose wait must run out; returns the launch status (read the workspace afterwards)."""
+    return int(load().vxl_selftest_bounded_wait(_ptr(workspace), int(limit_cycles), _stream(stream)))
 
 
 def _prefill_shape(q, k, out, scale, validate, force_general, gather4=False, step=0, prefix_len=0,

@@ -64,13 +64,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after about a second of polling (clock64 based), so a lost signal
 // ends in an error code, never in a hang.
 constexpr long long kWaitCycles = 2000000000ll;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - start > kWaitCycles) return false;
+        if (clock64() - start > limit) return false;
     }
 }
 

@@ -441,9 +441,29 @@ vxl_status launch_prefill_general(const PrefillParams &p, const vxl_shape *s, cu
     return cudaGetLastError() == cudaSuccess ? VXL_OK : VXL_ERR_CUDA;
 }
 
+// One warp waits, with the kernels' own bounded wait, on a barrier that nothing will ever complete.
+__global__ void bounded_wait_probe_kernel(WsHeader *hdr, long long limit_cycles)
+{
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) { mbar_init(smem_u32(&bar), 1); mbar_fence_init(); }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, limit_cycles);
+    if (!ok && threadIdx.x == 0) raise_status(hdr, VXL_ERR_TIMEOUT, 900);
+}
+
 }  // namespace
 
 extern "C" {
+
+vxl_status vxl_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream)
+{
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return VXL_ERR_WORKSPACE;
+    if (limit_cycles <= 0 || limit_cycles > 200000000ll) return VXL_ERR_INVALID_ARG;     // a tenth of a second at most
+    bounded_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<WsHeader *>(workspace),
+                                                                                   (long long)limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? VXL_OK : VXL_ERR_CUDA;
+}
+
 
 const char *vxl_status_str(vxl_status s)
 {

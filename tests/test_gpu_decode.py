@@ -363,3 +363,20 @@ def test_many_short_chunks(mode):
     """2048 chunks of 16 tokens: the ranking runs over more chunks than threads in a warp or a CTA row."""
     d = inputs.make_decode(B=2, T=32768, L=16, R=4, Hq=8, Hkv=2, D=64, seed=95, n_planted=3)
     check_decode(d, 37, sparse=(mode == "packed"))
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
+    """Failure path shared by every kernel: a bounded wait on a barrier nothing completes gives up after its
+    limit (two million clocks here, about a millisecond), the status word says so, and the next call works."""
+    d = inputs.make_decode(B=1, T=1024, L=128, R=16, Hq=8, Hkv=4, D=128, seed=19, n_planted=1)
+    q, k, v, off, ridx = gpu_tensors(d)
+    shape = vb._decode_shape(q, k, None, None, False)
+    ws = vb.new_workspace(vb.workspace_bytes(vb.VXL_OP_DECODE, shape, d.C, d.R, 2, d.L), "cuda")
+    assert vb.selftest_bounded_wait(ws, 2_000_000) == vb.VXL_OK           # the launch itself succeeds
+    assert vb.device_status(ws) == vb.VXL_ERR_TIMEOUT
+    assert vb.device_status(ws) == vb.VXL_OK                               # cleared by the read
+    res = vb.bilevel_decode_attn(q, k, v, off, ridx, 2, max_chunk_len=d.L, scale=d.scale, workspace=ws, return_scores=True)
+    torch.cuda.synchronize()
+    assert vb.device_status(ws) == vb.VXL_OK
+    want, _ = ref.decode(d.q[0], d.k[0], d.v[0], d.chunk_offsets, d.retained_idx, res["topk"][0].cpu().numpy(), d.scale)
+    check_close(res["out"][0], want, "decode after a reported timeout")

@@ -190,3 +190,11 @@ def test_host_prefill_rejects_bad_arguments(lib):
     ranged = _shape(B=1, T=1024, Hq=4, Hkv=2, D=128, q_strides=(1024 * 512, 512, 128), kv_strides=(1024 * 256, 256, 128),
                     block_begin=1, block_count=1)
     assert call(ranged) == vb.VXL_ERR_UNSUPPORTED
+
+
+def test_selftest_bounded_wait_rejects_bad_arguments(lib):
+    f = lib.vxl_selftest_bounded_wait
+    assert f(None, 1000, None) == vb.VXL_ERR_WORKSPACE
+    assert f(ctypes.c_void_p(0x20010), 1000, None) == vb.VXL_ERR_WORKSPACE
+    assert f(ctypes.c_void_p(0x20000), 0, None) == vb.VXL_ERR_INVALID_ARG
+    assert f(ctypes.c_void_p(0x20000), 10**12, None) == vb.VXL_ERR_INVALID_ARG        # no long waits on request
