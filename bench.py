@@ -294,7 +294,10 @@ def oracle_decode_full(qb, kb, vb_, off, ridx, scale, topk, bytes_seq, repeats=3
 def workload_config(sh, topks, dB):
     return {"workload": sh.name, "T": sh.T, "chunk_len": sh.L, "chunks": sh.C, "retained_per_chunk": sh.R,
             "Hq": sh.Hq, "Hkv": sh.Hkv, "D": sh.D, "out": "fp32",
-            "decode_workload": f"cfg5: cache 262144 tok = 128 chunks x 2048, R=128, k in {list(topks)}, batch {dB} and batch 1"}
+            "decode_workload": f"cfg5: cache 262144 tok = 128 chunks x 2048, R=128, k in {list(topks)}, batch {dB} and batch 1",
+            "l2": "no flush: every call's inputs exceed the 126 MB L2 (prefill q+k+v+out = %.1f GB, a batch decode call "
+                  "reads 0.5-0.8 GB); batch-1 decode calls rotate over %d distinct caches" %
+                  ((sh.T * sh.Hq * sh.D * 6 + 4 * sh.T * sh.Hkv * sh.D) / 1e9, dB)}
 
 
 def cpu_inputs(sh):
