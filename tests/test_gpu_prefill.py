@@ -369,3 +369,31 @@ def test_ragged_chunks_batched_bf16_out_and_range_fallback():
     want, _ = ref.prefill(cases[1].q, cases[1].k, cases[1].v, L, cases[0].retained_idx, cases[1].scale)
     check_close(out2[1, L:2 * L], want[L:2 * L], "ragged range call")
     assert torch.isnan(out2[:, :L]).all() and torch.isnan(out2[:, 2 * L:]).all()
+
+
+@pytest.mark.parametrize("T,L,R,Hq,Hkv,D", [
+    (16384, 2048, 128, 8, 2, 64),     # head dimension 64 over many work items per CTA
+    (16384, 64, 8, 4, 2, 64),         # the tiny configuration's chunk shape, 256 chunks of it
+    (24576, 192, 24, 7, 1, 128),      # 128 short ragged chunks, retained list of 127 x 24 rows
+])
+def test_head_dim_64_and_short_chunks_at_scale_sampled(T, L, R, Hq, Hkv, D):
+    case = inputs.make_prefill(T=T, L=L, R=R, Hq=Hq, Hkv=Hkv, D=D, seed=T + L + D, chunk_mean_std=0.5)
+    assert vb.prefill_kernel_kind(B=1, T=T, Hq=Hq, Hkv=Hkv, D=D, chunk_len=L, R=R) == 1
+    rows = sample_rows(T, L, 96, seed=L)
+    compare_sampled(case, rows)
+
+
+def test_head_dim_64_batched_bf16_out_with_window():
+    a = inputs.make_prefill_window(T_vis=1536, L=512, step=256, prefix_len=70, R=20, Hq=6, Hkv=2, D=64, seed=301)
+    b = inputs.make_prefill_window(T_vis=1536, L=512, step=256, prefix_len=70, R=20, Hq=6, Hkv=2, D=64, seed=302)
+    q = torch.stack([to_gpu(a.q), to_gpu(b.q)]); k = torch.stack([to_gpu(a.k), to_gpu(b.k)])
+    v = torch.stack([to_gpu(a.v), to_gpu(b.v)])
+    ridx = torch.from_numpy(a.retained_idx).cuda()
+    assert vb.prefill_kernel_kind(B=2, T=a.T, Hq=6, Hkv=2, D=64, chunk_len=512, R=20, step=256, prefix_len=70) == 1
+    out, lse = vb.chunk_prefill_attn(q, k, v, a.L, ridx, scale=a.scale, step=a.step, prefix_len=a.prefix_len,
+                                     out_dtype=torch.bfloat16, return_lse=True)
+    torch.cuda.synchronize()
+    for i, c in enumerate((a, b)):
+        want, want_lse = ref.prefill_window(c.q, c.k, c.v, c.L, c.step, c.prefix_len, a.retained_idx, c.scale)
+        check_close(out[i], want, f"D=64 batched window b{i}", max_err=2e-2, mean_err=2e-3)
+        check_close(lse[i], want_lse, "lse", max_err=LSE_ABS_ERR, mean_err=LSE_ABS_ERR)
