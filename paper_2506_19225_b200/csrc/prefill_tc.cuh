@@ -241,7 +241,7 @@ __host__ __device__ constexpr uint32_t tc_idesc(bool b_mn_major, uint32_t n = 12
 // Probabilities of columns [LO, HI) of one score row: p = 2^(s*scale - m), packed to bf16 pairs,
 // with two running partial sums.
 #ifndef VXL_TC_SPEC
-#define VXL_TC_SPEC 16
+#define VXL_TC_SPEC 32
 #endif
 constexpr int kTcSpec = VXL_TC_SPEC;                      // columns exponentiated ahead of the row max
 template <int LO, int HI>
